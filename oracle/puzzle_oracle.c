@@ -73,13 +73,16 @@ double oracle_e4m3_decode(uint8_t code) {
 }
 
 /* Nearest E4M3 code to y: round to nearest, ties to the code whose mantissa
- * LSB is 0, magnitudes above the largest finite value saturate to it, NaN
- * stays NaN, the sign of zero is kept.  Done as a search over the codebook. */
+ * LSB is 0, magnitudes above the largest finite value saturate to it, the sign
+ * of zero is kept.  Every NaN maps to the one canonical NaN code 0x7F: the
+ * sign a NaN carries out of a division is not fixed by IEEE 754 (it differs
+ * between processors), so it cannot be part of a bit-exact contract.
+ * Done as a search over the codebook. */
 uint8_t oracle_e4m3_encode(float y) {
   uint8_t sign = signbit(y) ? 0x80 : 0x00;
   double a = fabs((double)y);
   int lo;
-  if (isnan(y)) return (uint8_t)(sign | 0x7F);
+  if (isnan(y)) return (uint8_t)0x7F;
   if (a >= oracle_e4m3_decode(0x7E)) return (uint8_t)(sign | 0x7E);
   /* magnitudes of codes 0x00..0x7E increase strictly with the code */
   lo = 0;
