@@ -1,0 +1,156 @@
+/*
+ * puzzle_attn.h -- C ABI of the FP8-KV decode-attention library (sm_100a).
+ *
+ * One decode step of one attention layer of a gpt-oss-style grouped-query
+ * model, as the paper's serving optimisations shape it:
+ *
+ *   - the KV cache is stored as FP8 (E4M3) with max-calibrated dequantisation
+ *     scales (paper, Section "KV Quantization"); a bf16 cache is the comparison
+ *     variant the paper measures against;
+ *   - every layer is either full-context attention or window attention that
+ *     sees only the most recent W tokens (paper, Section "Window attention for
+ *     long-context inference"); which layers are which is the per-layer choice
+ *     the architecture search makes (Section "Puzzle Optimization", "Blocks,
+ *     subblocks, and search space");
+ *   - decode is KV-cache-I/O bound (Section "Optimized Scenarios"), so the
+ *     library streams every visible K/V byte exactly once per step.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller, unless marked
+ *     "host".  The two descriptor structs are read on the host during the call.
+ *   - Nothing is allocated, freed or kept between calls.  Work is enqueued on
+ *     the CUDA stream passed as `stream` (a cudaStream_t cast to void*; NULL is
+ *     the default stream) and the call returns without synchronising.
+ *   - Errors that the host can see (NULL required pointer, unsupported shape,
+ *     workspace too small) return a code BEFORE anything is launched.  A CUDA
+ *     launch error maps to PUZZLE_ERR_CUDA.  Errors only the device can see
+ *     (a block-table entry outside [0, num_blocks), a sequence longer than its
+ *     table row) set a bit in *dev_status, skip the access and never trap.
+ *   - Shapes supported by this version: head_dim 64, block_size 16,
+ *     num_q_heads == 8 * num_kv_heads, batch <= 4096.
+ *
+ * Cache layout (both K and V):  [num_blocks][num_kv_heads][block_size][head_dim]
+ *   elements u8 (E4M3 codes) or bf16; one (block, KV head) is 1 KiB (FP8) or
+ *   2 KiB (bf16) contiguous.  Base pointers must be 16-byte aligned.
+ */
+#ifndef PUZZLE_ATTN_H_
+#define PUZZLE_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define PUZZLE_API __attribute__((visibility("default")))
+#else
+#define PUZZLE_API
+#endif
+
+typedef enum {
+  PUZZLE_OK = 0,
+  PUZZLE_ERR_NULL = 1,        /* a required pointer is NULL */
+  PUZZLE_ERR_SHAPE = 2,       /* sizes inconsistent or out of range */
+  PUZZLE_ERR_UNSUPPORTED = 3, /* valid but not built in this version */
+  PUZZLE_ERR_WORKSPACE = 4,   /* workspace missing or too small */
+  PUZZLE_ERR_CUDA = 5         /* a CUDA call or launch failed */
+} puzzle_status;
+
+typedef enum { PUZZLE_KV_FP8_E4M3 = 0, PUZZLE_KV_BF16 = 1 } puzzle_kv_dtype;
+
+/* bits of *dev_status */
+#define PUZZLE_DEV_BAD_BLOCK 1u  /* block-table entry outside [0, num_blocks) */
+#define PUZZLE_DEV_SEQ_TOO_LONG 2u /* seq_len > max_blocks_per_seq * block_size (clamped) */
+#define PUZZLE_DEV_WAIT_EXPIRED 4u /* a bounded wait on a copy ran out; results invalid */
+
+/* One per layer: the layer's attention choice (host struct). */
+typedef struct {
+  int32_t num_q_heads;  /* 64 */
+  int32_t num_kv_heads; /* 8; consecutive groups of 8 query heads share one KV head */
+  int32_t head_dim;     /* 64 */
+  int32_t block_size;   /* 16 tokens per cache block */
+  int32_t window;       /* 0 = full context; W > 0 = the W most recent tokens, current one included */
+  int32_t kv_dtype;     /* puzzle_kv_dtype */
+  float sm_scale;       /* logit scale, 1/sqrt(head_dim) */
+} puzzle_layer_desc;
+
+/* One per layer: that layer's cache and how this batch maps onto it (host
+ * struct holding device pointers). */
+typedef struct {
+  void* k_cache;              /* see "Cache layout" */
+  void* v_cache;
+  int64_t num_blocks;
+  const int32_t* block_table; /* [batch][max_blocks_per_seq]; NULL = contiguous: block = b*max_blocks_per_seq + i.
+                                 Entries for blocks that lie wholly outside the visible range are never read. */
+  int32_t max_blocks_per_seq;
+  const int32_t* seq_lens;    /* [batch], length AFTER this step's append; 0 is legal */
+  const float* k_scale;       /* [num_kv_heads] dequantisation scales (x ~= code * scale); NULL = 1; FP8 only */
+  const float* v_scale;
+} puzzle_kv_view;
+
+/* Quantise-and-append of the new token's K and V (one token per sequence).
+ * FP8: code = E4M3(round-to-nearest-even, saturating at +-448, of the float32
+ * quotient x / scale[h]); NaN -> 0x7F.  bf16: the value is copied.  The token
+ * lands at logical position seq_lens[b]-1 through the block table.  This is
+ * the FP8 KV quantisation of Section "KV Quantization" applied at decode time.
+ *   k_new, v_new: bf16 [batch][num_kv_heads][head_dim].
+ *   dev_status: optional int32 device word, bits OR-ed in on device-side errors. */
+PUZZLE_API puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* k_new,
+                               const void* v_new, int32_t batch, int32_t* dev_status, void* stream);
+
+/* Bytes of scratch puzzle_decode_attn needs for this batch and split choice
+ * (0 on invalid arguments).  num_splits == 0 selects the balanced schedule. */
+PUZZLE_API size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits);
+
+/* Decode-step attention of one layer: for every sequence b and query head g
+ * (KV head h = g / 8), over the visible keys j in [L - min(W, L), L) with
+ * L = seq_lens[b] (all of [0, L) when window == 0):
+ *     s_j = sm_scale * k_scale[h] * (q_g . Kcode_j),  M = max(max_j s_j, sink_g),
+ *     Z = e^(sink_g - M) + sum_j e^(s_j - M),  out = v_scale[h] * sum_j e^(s_j - M) Vcode_j / Z.
+ * Full vs window is the paper's per-layer choice (Section "Window attention for
+ * long-context inference"); the sink is one extra softmax column per query head
+ * that carries no value.  Internally: a split-KV pass that writes float32
+ * partial (o, lse) into the workspace, then a log-sum-exp merge.
+ *   q: bf16 [batch][num_q_heads][head_dim];  sinks: float32 [num_q_heads] or NULL (no sink);
+ *   out: bf16 [batch][num_q_heads][head_dim];  lse_out: float32 [batch][num_q_heads] or NULL;
+ *   num_splits: 0 = balanced schedule (recommended); S >= 1 = every (sequence, KV head) context is
+ *     cut into S equal runs of 64-token tiles;
+ *   workspace: device scratch of at least puzzle_decode_attn_workspace_bytes(...) bytes, 16-byte
+ *     aligned, contents undefined before and after;
+ *   dev_status: optional int32 device word (see PUZZLE_DEV_*).
+ * An empty context gives out = 0 and lse = sink (-inf without a sink). */
+PUZZLE_API puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                 const float* sinks, void* out, float* lse_out, int32_t batch,
+                                 int32_t num_splits, void* workspace, size_t workspace_bytes,
+                                 int32_t* dev_status, void* stream);
+
+/* Log-sum-exp merge of partial attention results (the second phase above, also
+ * usable on partials that came from elsewhere, e.g. context shards on other
+ * GPUs).  For every row r = (b, g):
+ *     M = max(sink_g, max_p lse_p),  Z = e^(sink_g - M) + sum_p e^(lse_p - M),
+ *     out = sum_p e^(lse_p - M) o_p / Z,  lse_out = M + ln Z.
+ *   part_o: float32 [batch][Hq][S][D];  part_lse: float32 [batch][Hq][S] (natural log; -inf = empty part);
+ *   num_parts: int32 [batch] or NULL (= S for all);  sinks: float32 [Hq] or NULL;
+ *   out: bf16 [batch][Hq][D];  lse_out: float32 [batch][Hq] or NULL.  D must be a multiple of 64, <= 512. */
+PUZZLE_API puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, const int32_t* num_parts,
+                                const float* sinks, void* out, float* lse_out, int32_t batch, int32_t Hq,
+                                int32_t D, int32_t S, void* stream);
+
+/* Read-only streaming pass over `bytes` bytes at `buf` (16-byte aligned,
+ * bytes a multiple of 16): the XOR of all words is written to *sink (device,
+ * 8 bytes).  Not part of the method; it measures the read bandwidth the
+ * attention kernel is bounded by on the device it runs on. */
+PUZZLE_API puzzle_status puzzle_hbm_read_probe(const void* buf, size_t bytes, uint64_t* sink, void* stream);
+
+/* Static description of a status code (host string, never NULL). */
+PUZZLE_API const char* puzzle_status_string(puzzle_status s);
+
+/* Number of kernels this library has launched from this process so far. */
+PUZZLE_API int64_t puzzle_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PUZZLE_ATTN_H_ */

@@ -1,0 +1,26 @@
+"""B200-native FP8-KV decode attention (split-KV + merge) and fused FP8 KV append.
+
+The compute runs in ``lib/libpuzzle_attn.so`` (hand-written sm_100a kernels behind a C ABI,
+declared in ``include/puzzle_attn.h``).  This package only marshals torch tensors into that
+ABI; there is no Python or CPU fallback: a missing library raises.
+"""
+from .binding import (  # noqa: F401
+    KV_BF16,
+    KV_FP8_E4M3,
+    DEV_BAD_BLOCK,
+    DEV_SEQ_TOO_LONG,
+    DEV_WAIT_EXPIRED,
+    KVView,
+    LayerDesc,
+    PuzzleError,
+    kv_view,
+    layer_desc,
+    library_path,
+    puzzle_attn_merge,
+    puzzle_decode_attn,
+    puzzle_decode_attn_workspace_bytes,
+    puzzle_hbm_read_probe,
+    puzzle_kv_append,
+    puzzle_launch_count,
+    puzzle_status_string,
+)

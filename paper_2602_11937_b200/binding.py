@@ -1,0 +1,179 @@
+"""ctypes binding of the C ABI: same entry-point names, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "lib", "libpuzzle_attn.so")
+_lib = None
+
+KV_FP8_E4M3 = 0
+KV_BF16 = 1
+DEV_BAD_BLOCK = 1
+DEV_SEQ_TOO_LONG = 2
+DEV_WAIT_EXPIRED = 4
+
+EXPORTS = (
+    "puzzle_kv_append",
+    "puzzle_decode_attn_workspace_bytes",
+    "puzzle_decode_attn",
+    "puzzle_attn_merge",
+    "puzzle_hbm_read_probe",
+    "puzzle_status_string",
+    "puzzle_launch_count",
+)
+
+
+class PuzzleError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: status %d (%s)" % (where, code, puzzle_status_string(code)))
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("block_size", ctypes.c_int32), ("window", ctypes.c_int32), ("kv_dtype", ctypes.c_int32),
+                ("sm_scale", ctypes.c_float)]
+
+
+class KVView(ctypes.Structure):
+    _fields_ = [("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p), ("num_blocks", ctypes.c_int64),
+                ("block_table", ctypes.c_void_p), ("max_blocks_per_seq", ctypes.c_int32),
+                ("seq_lens", ctypes.c_void_p), ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                "CUDA library %s is missing: build it with `python -m paper_2602_11937_b200.build` "
+                "(there is no CPU fallback)" % _LIB_PATH)
+        lib = ctypes.CDLL(_LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        lib.puzzle_kv_append.restype = ctypes.c_int
+        lib.puzzle_kv_append.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, i32, vp, vp]
+        lib.puzzle_decode_attn_workspace_bytes.restype = sz
+        lib.puzzle_decode_attn_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32, i32]
+        lib.puzzle_decode_attn.restype = ctypes.c_int
+        lib.puzzle_decode_attn.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp, i32, i32,
+                                           vp, sz, vp, vp]
+        lib.puzzle_attn_merge.restype = ctypes.c_int
+        lib.puzzle_attn_merge.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
+        lib.puzzle_hbm_read_probe.restype = ctypes.c_int
+        lib.puzzle_hbm_read_probe.argtypes = [vp, sz, vp, vp]
+        lib.puzzle_status_string.restype = ctypes.c_char_p
+        lib.puzzle_status_string.argtypes = [ctypes.c_int]
+        lib.puzzle_launch_count.restype = ctypes.c_int64
+        lib.puzzle_launch_count.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def _p(t: Optional[torch.Tensor], dtype=None, name="tensor"):
+    """Device pointer of a contiguous CUDA tensor (None -> NULL)."""
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor" % name)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("%s must be %s, got %s" % (name, dtype, t.dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def layer_desc(window: int = 0, kv_dtype: int = KV_FP8_E4M3, num_q_heads: int = 64, num_kv_heads: int = 8,
+               head_dim: int = 64, block_size: int = 16, sm_scale: Optional[float] = None) -> LayerDesc:
+    return LayerDesc(num_q_heads, num_kv_heads, head_dim, block_size, int(window), int(kv_dtype),
+                     float(sm_scale if sm_scale is not None else head_dim ** -0.5))
+
+
+def kv_view(k_cache: torch.Tensor, v_cache: torch.Tensor, seq_lens: torch.Tensor,
+            block_table: Optional[torch.Tensor] = None, max_blocks_per_seq: Optional[int] = None,
+            k_scale: Optional[torch.Tensor] = None, v_scale: Optional[torch.Tensor] = None) -> KVView:
+    """Describe one layer's cache ([num_blocks][Hkv][16][D], uint8 codes or bf16) for this batch.
+
+    The view holds raw pointers: keep the tensors alive while it is in use."""
+    if block_table is not None:
+        max_blocks_per_seq = block_table.shape[1]
+    if max_blocks_per_seq is None:
+        raise ValueError("max_blocks_per_seq is required without a block table")
+    v = KVView()
+    v.k_cache = k_cache.data_ptr() if k_cache.is_cuda and k_cache.is_contiguous() else None
+    v.v_cache = v_cache.data_ptr() if v_cache.is_cuda and v_cache.is_contiguous() else None
+    v.num_blocks = k_cache.shape[0]
+    v.block_table = _p(block_table, torch.int32, "block_table")
+    v.max_blocks_per_seq = int(max_blocks_per_seq)
+    v.seq_lens = _p(seq_lens, torch.int32, "seq_lens")
+    v.k_scale = _p(k_scale, torch.float32, "k_scale")
+    v.v_scale = _p(v_scale, torch.float32, "v_scale")
+    return v
+
+
+def puzzle_status_string(code: int) -> str:
+    return _load().puzzle_status_string(int(code)).decode()
+
+
+def puzzle_launch_count() -> int:
+    return int(_load().puzzle_launch_count())
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise PuzzleError(code, where)
+
+
+def puzzle_kv_append(desc: LayerDesc, view: KVView, k_new: torch.Tensor, v_new: torch.Tensor,
+                     dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    batch = k_new.shape[0]
+    _check(_load().puzzle_kv_append(ctypes.byref(desc), ctypes.byref(view), _p(k_new, torch.bfloat16, "k_new"),
+                                    _p(v_new, torch.bfloat16, "v_new"), batch, _p(dev_status, torch.int32),
+                                    _stream(stream)), "puzzle_kv_append")
+
+
+def puzzle_decode_attn_workspace_bytes(desc: LayerDesc, batch: int, num_splits: int = 0) -> int:
+    return int(_load().puzzle_decode_attn_workspace_bytes(ctypes.byref(desc), int(batch), int(num_splits)))
+
+
+def puzzle_decode_attn(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Optional[torch.Tensor],
+                       out: torch.Tensor, lse_out: Optional[torch.Tensor] = None, num_splits: int = 0,
+                       workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                       stream=None) -> None:
+    batch = q.shape[0]
+    if workspace is None:
+        raise ValueError("workspace is required (size it with puzzle_decode_attn_workspace_bytes)")
+    _check(_load().puzzle_decode_attn(ctypes.byref(desc), ctypes.byref(view), _p(q, torch.bfloat16, "q"),
+                                      _p(sinks, torch.float32, "sinks"), _p(out, torch.bfloat16, "out"),
+                                      _p(lse_out, torch.float32, "lse_out"), batch, int(num_splits), _p(workspace),
+                                      workspace.numel() * workspace.element_size(), _p(dev_status, torch.int32),
+                                      _stream(stream)), "puzzle_decode_attn")
+
+
+def puzzle_attn_merge(part_o: torch.Tensor, part_lse: torch.Tensor, num_parts: Optional[torch.Tensor],
+                      sinks: Optional[torch.Tensor], out: torch.Tensor, lse_out: Optional[torch.Tensor] = None,
+                      stream=None) -> None:
+    batch, hq, s, d = part_o.shape
+    _check(_load().puzzle_attn_merge(_p(part_o, torch.float32, "part_o"), _p(part_lse, torch.float32, "part_lse"),
+                                     _p(num_parts, torch.int32, "num_parts"), _p(sinks, torch.float32, "sinks"),
+                                     _p(out, torch.bfloat16, "out"), _p(lse_out, torch.float32, "lse_out"),
+                                     batch, hq, d, s, _stream(stream)), "puzzle_attn_merge")
+
+
+def puzzle_hbm_read_probe(buf: torch.Tensor, sink: torch.Tensor, stream=None) -> None:
+    _check(_load().puzzle_hbm_read_probe(_p(buf), buf.numel() * buf.element_size(), _p(sink), _stream(stream)),
+           "puzzle_hbm_read_probe")

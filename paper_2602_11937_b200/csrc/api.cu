@@ -1,0 +1,249 @@
+// Host side of the C ABI declared in include/puzzle_attn.h: argument checks, TMA descriptor
+// encoding and kernel launches.  No allocation, no synchronisation, no state besides a launch counter.
+#include <atomic>
+#include <cstring>
+
+#include "common.cuh"
+#include "decode_attn.cuh"
+
+namespace puzzle {
+
+static std::atomic<long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+struct DeviceInfo {
+  int sm_count = 0;
+  bool smem_set_fp8 = false;
+};
+DeviceInfo& device_info() {
+  static DeviceInfo info[64];
+  int dev = 0;
+  cudaGetDevice(&dev);
+  DeviceInfo& d = info[dev & 63];
+  if (d.sm_count == 0) cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev);
+  return d;
+}
+
+puzzle_status check_desc(const puzzle_layer_desc* d) {
+  if (!d) return PUZZLE_ERR_NULL;
+  if (d->num_q_heads <= 0 || d->num_kv_heads <= 0 || d->head_dim <= 0 || d->block_size <= 0 || d->window < 0)
+    return PUZZLE_ERR_SHAPE;
+  if (d->num_q_heads % d->num_kv_heads != 0) return PUZZLE_ERR_SHAPE;
+  if (d->kv_dtype != PUZZLE_KV_FP8_E4M3 && d->kv_dtype != PUZZLE_KV_BF16) return PUZZLE_ERR_SHAPE;
+  if (d->head_dim != kHeadDim || d->block_size != kBlock || d->num_q_heads != kGroup * d->num_kv_heads)
+    return PUZZLE_ERR_UNSUPPORTED;
+  return PUZZLE_OK;
+}
+
+puzzle_status check_view(const puzzle_layer_desc* d, const puzzle_kv_view* kv, int batch) {
+  if (!kv || !kv->k_cache || !kv->v_cache || !kv->seq_lens) return PUZZLE_ERR_NULL;
+  if (batch <= 0 || kv->num_blocks <= 0 || kv->max_blocks_per_seq <= 0) return PUZZLE_ERR_SHAPE;
+  if (batch > kMaxBatch) return PUZZLE_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(kv->k_cache) & 15) || (reinterpret_cast<uintptr_t>(kv->v_cache) & 15))
+    return PUZZLE_ERR_SHAPE;
+  // rows of the 2-D view of the cache must fit a signed 32-bit TMA coordinate
+  if (kv->num_blocks * d->num_kv_heads * (long long)kBlock >= (1ll << 31) - 64) return PUZZLE_ERR_UNSUPPORTED;
+  if (!kv->block_table && (long long)batch * kv->max_blocks_per_seq > kv->num_blocks) return PUZZLE_ERR_SHAPE;
+  return PUZZLE_OK;
+}
+
+// 2-D view of a cache: rows = (block, kv head, slot), one row = one token's head_dim elements.
+// Box = one 16-token block of one KV head; swizzle spans one row (64 B for FP8, 128 B for bf16).
+bool make_cache_map(CUtensorMap* m, void* base, long long rows, int elem_bytes) {
+  EncodeTiledFn enc = encode_tiled();
+  if (!enc) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * elem_bytes};
+  const cuuint32_t box[2] = {(cuuint32_t)kHeadDim, (cuuint32_t)kBlock};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base,
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   elem_bytes == 1 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int grid_ctas() { return device_info().sm_count > 0 ? device_info().sm_count : 1; }
+
+size_t workspace_floats(int batch, int Hkv, int num_splits) {
+  const size_t rows = num_splits == 0 ? ((size_t)grid_ctas() * kWarps + (size_t)batch * Hkv) * kGroup
+                                      : (size_t)batch * Hkv * kGroup * num_splits;
+  return rows * (kHeadDim + 1);
+}
+
+}  // namespace
+}  // namespace puzzle
+
+using namespace puzzle;
+
+extern "C" {
+
+const char* puzzle_status_string(puzzle_status s) {
+  switch (s) {
+    case PUZZLE_OK: return "ok";
+    case PUZZLE_ERR_NULL: return "a required pointer is NULL";
+    case PUZZLE_ERR_SHAPE: return "inconsistent or out-of-range sizes";
+    case PUZZLE_ERR_UNSUPPORTED: return "shape or dtype not supported by this build";
+    case PUZZLE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case PUZZLE_ERR_CUDA: return "a CUDA call or kernel launch failed";
+  }
+  return "unknown status";
+}
+
+int64_t puzzle_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* k_new,
+                               const void* v_new, int32_t batch, int32_t* dev_status, void* stream) {
+  puzzle_status st = check_desc(desc);
+  if (st != PUZZLE_OK) return st;
+  st = check_view(desc, kv, batch);
+  if (st != PUZZLE_OK) return st;
+  if (!k_new || !v_new) return PUZZLE_ERR_NULL;
+  const long long threads = 2ll * batch * desc->num_kv_heads * (kHeadDim / 2);
+  const int grid = (int)((threads + 255) / 256);
+  kv_append_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      kv->k_cache, kv->v_cache, static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+      kv->block_table, kv->seq_lens, kv->k_scale, kv->v_scale, kv->num_blocks, batch, desc->num_kv_heads,
+      kv->max_blocks_per_seq, desc->kv_dtype, dev_status);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+}
+
+size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits) {
+  if (check_desc(desc) != PUZZLE_OK || batch <= 0 || batch > kMaxBatch || num_splits < 0) return 0;
+  return workspace_floats(batch, desc->num_kv_heads, num_splits) * sizeof(float);
+}
+
+puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                 const float* sinks, void* out, float* lse_out, int32_t batch, int32_t num_splits,
+                                 void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+  puzzle_status st = check_desc(desc);
+  if (st != PUZZLE_OK) return st;
+  st = check_view(desc, kv, batch);
+  if (st != PUZZLE_OK) return st;
+  if (!q || !out) return PUZZLE_ERR_NULL;
+  if (num_splits < 0 || num_splits > 65536) return PUZZLE_ERR_SHAPE;
+  if (desc->kv_dtype != PUZZLE_KV_FP8_E4M3) return PUZZLE_ERR_UNSUPPORTED;
+  const int Hkv = desc->num_kv_heads;
+  const size_t need = workspace_floats(batch, Hkv, num_splits) * sizeof(float);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 15)) return PUZZLE_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  const int ctas = grid_ctas();
+  const size_t rows = need / sizeof(float) / (kHeadDim + 1);
+  float* part_o = static_cast<float*>(workspace);
+  float* part_lse = part_o + rows * kHeadDim;
+
+  DecodeParams P;
+  std::memset(&P, 0, sizeof P);
+  const long long cache_rows = kv->num_blocks * Hkv * (long long)kBlock;
+  if (!make_cache_map(&P.tmK, kv->k_cache, cache_rows, 1) || !make_cache_map(&P.tmV, kv->v_cache, cache_rows, 1))
+    return PUZZLE_ERR_CUDA;
+  P.q = static_cast<const __nv_bfloat16*>(q);
+  P.block_table = kv->block_table;
+  P.seq_lens = kv->seq_lens;
+  P.k_scale = kv->k_scale;
+  P.v_scale = kv->v_scale;
+  P.part_o = part_o;
+  P.part_lse = part_lse;
+  P.dev_status = dev_status;
+  P.num_blocks = kv->num_blocks;
+  P.batch = batch;
+  P.Hkv = Hkv;
+  P.max_blocks_per_seq = kv->max_blocks_per_seq;
+  P.window = desc->window;
+  P.num_splits = num_splits;
+  P.oob_row = (int)cache_rows;
+  P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
+
+  const size_t smem = decode_attn_fp8_smem_bytes(batch);
+  DeviceInfo& di = device_info();
+  if (!di.smem_set_fp8) {
+    if (cudaFuncSetAttribute(decode_attn_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)decode_attn_fp8_smem_bytes(kMaxBatch)) != cudaSuccess)
+      return PUZZLE_ERR_CUDA;
+    di.smem_set_fp8 = true;
+  }
+  decode_attn_fp8_kernel<<<ctas, kWarps * 32, smem, s>>>(P);
+  count_launch();
+  if (cudaGetLastError() != cudaSuccess) return PUZZLE_ERR_CUDA;
+
+  MergeParams M;
+  std::memset(&M, 0, sizeof M);
+  M.part_o = part_o;
+  M.part_lse = part_lse;
+  M.sinks = sinks;
+  M.out = static_cast<__nv_bfloat16*>(out);
+  M.lse_out = lse_out;
+  M.batch = batch;
+  M.Hq = desc->num_q_heads;
+  M.D = kHeadDim;
+  M.S = num_splits;
+  M.balanced = num_splits == 0;
+  M.seq_lens = kv->seq_lens;
+  M.Hkv = Hkv;
+  M.window = desc->window;
+  M.max_tokens = kv->max_blocks_per_seq * kBlock;
+  M.num_workers = ctas * kWarps;
+  const long long mrows = (long long)batch * desc->num_q_heads;
+  attn_merge_kernel<<<(unsigned)((mrows + kWarps - 1) / kWarps), kWarps * 32, attn_merge_smem_bytes(batch, M.balanced),
+                      s>>>(M);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+}
+
+puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, const int32_t* num_parts,
+                                const float* sinks, void* out, float* lse_out, int32_t batch, int32_t Hq, int32_t D,
+                                int32_t S, void* stream) {
+  if (!part_o || !part_lse || !out) return PUZZLE_ERR_NULL;
+  if (batch <= 0 || Hq <= 0 || S <= 0 || D <= 0) return PUZZLE_ERR_SHAPE;
+  if (D % 64 != 0 || D > 512) return PUZZLE_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(part_o) & 7) || (reinterpret_cast<uintptr_t>(out) & 3)) return PUZZLE_ERR_SHAPE;
+  MergeParams M;
+  std::memset(&M, 0, sizeof M);
+  M.part_o = part_o;
+  M.part_lse = part_lse;
+  M.num_parts = num_parts;
+  M.sinks = sinks;
+  M.out = static_cast<__nv_bfloat16*>(out);
+  M.lse_out = lse_out;
+  M.batch = batch;
+  M.Hq = Hq;
+  M.D = D;
+  M.S = S;
+  M.balanced = 0;
+  const long long rows = (long long)batch * Hq;
+  attn_merge_kernel<<<(unsigned)((rows + kWarps - 1) / kWarps), kWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(M);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+}
+
+puzzle_status puzzle_hbm_read_probe(const void* buf, size_t bytes, uint64_t* sink, void* stream) {
+  if (!buf || !sink) return PUZZLE_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(buf) & 15) || (bytes & 15) || bytes == 0) return PUZZLE_ERR_SHAPE;
+  const int ctas = grid_ctas() * 4;
+  hbm_read_probe_kernel<<<ctas, 512, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const uint4*>(buf), bytes / 16, reinterpret_cast<unsigned long long*>(sink));
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -109,6 +109,12 @@ def workload(config_id: int, scale: float = 1.0, pattern: str = "parent") -> Wor
     raise ValueError("config_id must be 1..5")
 
 
+def bf16_bits(t: torch.Tensor):
+    """bf16 tensor -> numpy uint16 bit patterns (numpy has no bf16 type)."""
+    import numpy as np
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
 # ------------------------------------------------------------------ draws ---
 
 def draw_q(w: Workload, layer: int = 0, device: str = "cpu") -> torch.Tensor:

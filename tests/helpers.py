@@ -13,9 +13,7 @@ import oracle
 import synth
 
 
-def bf16_bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor -> uint16 bit patterns (numpy has no bf16)."""
-    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+bf16_bits = synth.bf16_bits
 
 
 def bits_to_bf16(a: np.ndarray) -> torch.Tensor:

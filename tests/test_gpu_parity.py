@@ -1,0 +1,284 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle,
+element by element on the same seeded inputs.
+
+Bars: appended FP8 bytes bit-exact; attention output max |err| <= 2e-3 (bf16 output,
+N(0,1) inputs).  Where |out| reaches 1 and beyond, one bf16 half-ulp (2^-8 |ref|) is
+added, because no bf16 value is closer than that (see gpu_helpers.error_bound).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from helpers import bf16_bits, bf16_bits_to_f64, make_case, oracle_append, oracle_attn
+
+pytestmark = pytest.mark.gpu
+
+
+def _dev(case):
+    from gpu_helpers import DeviceCase
+    return DeviceCase(case)
+
+
+# ------------------------------------------------------------------ append ---
+
+@pytest.mark.parametrize("scale_kind", ["one", "pow2", "amax"])
+def test_append_all_bf16_patterns_bit_exact(scale_kind):
+    bits = np.arange(65536, dtype=np.uint16)
+    w = synth.Workload("all_bf16", 1, 65536 // (8 * 64), 16, [0], paged=False)
+    nb = w.batch * w.blocks_per_seq
+    scale = {"one": np.ones(8, np.float32), "pow2": np.full(8, 2.0 ** -3, np.float32),
+             "amax": (np.linspace(0.7, 5.3, 8) / 448).astype(np.float32)}[scale_kind]
+    case = dict(w=w, kv_dtype=oracle.KV_FP8_E4M3, num_blocks=nb,
+                k_cache=np.full((nb, 8, 16, 64), 0xA5, np.uint8), v_cache=np.full((nb, 8, 16, 64), 0x5A, np.uint8),
+                table=None, seq_lens=np.full(w.batch, 7, np.int32), k_scale=scale, v_scale=scale[::-1].copy(),
+                q=np.zeros((w.batch, 64, 64), np.uint16), sinks=np.zeros(64, np.float32),
+                k_new=bits.reshape(w.batch, 8, 64), v_new=bits[::-1].reshape(w.batch, 8, 64).copy(), sm_scale=0.125)
+    dev = _dev(case)
+    dev.append()
+    oracle_append(case)
+    gk, gv = dev.cache_bytes()
+    assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
+    assert int(dev.status.item()) == 0
+
+
+def test_append_null_scales_means_one():
+    w = synth.workload(1, scale=0.25)
+    case = make_case(w, no_scales=True)
+    ref = dict(case)
+    case = dict(case, k_scale=None, v_scale=None)
+    dev = _dev(case)
+    dev.append()
+    oracle_append(ref)
+    gk, gv = dev.cache_bytes()
+    assert np.array_equal(gk, ref["k_cache"]) and np.array_equal(gv, ref["v_cache"])
+
+
+@pytest.mark.parametrize("cfg,scale", [(1, 1.0), (2, 0.1), (4, 0.02)])
+def test_append_paged_scatter_bit_exact(cfg, scale):
+    w = synth.workload(cfg, scale=scale)
+    lens = synth.draw_seq_lens(w).numpy().copy()
+    lens[0] = 1
+    if w.batch > 2:
+        lens[1], lens[2] = 16, 17
+    if w.batch > 3:
+        lens[3] = 0  # an empty sequence appends nothing
+    case = make_case(w, seq_lens=lens)
+    dev = _dev(case)
+    dev.append()
+    oracle_append(case)
+    gk, gv = dev.cache_bytes()
+    assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
+
+
+def test_append_bf16_cache_is_a_copy():
+    w = synth.workload(2, scale=0.05)
+    case = make_case(w, kv_dtype=oracle.KV_BF16)
+    dev = _dev(case)
+    dev.append()
+    oracle_append(case)
+    gk, gv = dev.cache_bytes()
+    assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
+
+
+# --------------------------------------------------------------- attention ---
+
+def _run_and_compare(case, window, num_splits=0, rel=False, sinks="case"):
+    from gpu_helpers import assert_close
+    dev = _dev(case)
+    dev.append()
+    oracle_append(case)
+    gk, gv = dev.cache_bytes()
+    assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
+    got, got_lse = dev.attn(window=window, num_splits=num_splits, sinks=sinks)
+    s = case["sinks"] if isinstance(sinks, str) else (None if sinks is None else sinks.cpu().numpy())
+    ref, ref_lse = oracle_attn(case, window, sinks=s)
+    assert int(dev.status.item()) == 0
+    err = assert_close(got, ref, "out W=%d S=%d" % (window, num_splits), rel=rel)
+    fin = np.isfinite(ref_lse)
+    assert np.array_equal(np.isfinite(got_lse), fin)
+    assert np.all(np.abs(got_lse[fin] - ref_lse[fin]) <= 2e-3)
+    return err
+
+
+def test_config1_full_contiguous():
+    _run_and_compare(make_case(synth.workload(1)), 0)
+
+
+@pytest.mark.parametrize("window", [0, 128])
+def test_config2_paged_full_and_window(window):
+    w = synth.workload(2, scale=0.25)          # batch 8, context 2048, scales from a 512-token prefix
+    layer = 0 if window == 0 else 1
+    _run_and_compare(make_case(w, layer=layer), window)
+
+
+@pytest.mark.parametrize("num_splits", [0, 8, 16, 128])
+def test_config3_scaled_kv_split_sweep(num_splits):
+    w = synth.workload(3, scale=0.125)         # batch 2, context 8192, K/V scaled per head by U[0.5, 4]
+    _run_and_compare(make_case(w), 0, num_splits=num_splits)
+
+
+@pytest.mark.parametrize("layer,window", [(0, 128), (1, 0), (2, 1000)])
+def test_config4_ragged_layers(layer, window):
+    w = synth.workload(4, scale=0.05)          # batch 3, ragged contexts up to 2458
+    _run_and_compare(make_case(w, layer=layer), window)
+
+
+def test_config5_long_context_fp8():
+    w = synth.workload(5, scale=0.04)          # batch 1 (rounded), context 5243
+    w.batch = 2
+    _run_and_compare(make_case(w, layer=1), 0)
+    _run_and_compare(make_case(w, layer=0), 128)
+
+
+EDGE_LENS = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200]
+
+
+@pytest.mark.parametrize("window", [0, 1, 16, 17, 100, 1000])
+@pytest.mark.parametrize("num_splits", [0, 1, 3])
+def test_edge_lengths_with_poisoned_tail(window, num_splits):
+    w = synth.Workload("edges", 1, len(EDGE_LENS), 200, [0], paged=True)
+    case = make_case(w, seq_lens=EDGE_LENS, poison_tail=True)
+    _run_and_compare(case, window, num_splits=num_splits)
+
+
+def test_no_sinks_and_empty_context():
+    from gpu_helpers import assert_close
+    w = synth.Workload("nosink", 1, 4, 90, [0], paged=True)
+    case = make_case(w, seq_lens=[90, 0, 1, 64])
+    dev = _dev(case)
+    dev.append(); oracle_append(case)
+    got, lse = dev.attn(window=0, sinks=None)
+    ref, ref_lse = oracle_attn(case, 0, sinks=None)
+    assert_close(got, ref, "no sinks")
+    assert np.all(np.isneginf(lse[1])) and not got[1].any()
+    # with sinks the empty sequence returns zeros and lse = sink
+    got, lse = dev.attn(window=0)
+    assert not got[1].any() and np.allclose(lse[1], case["sinks"], atol=1e-6)
+
+
+def test_no_scales_and_pow2_scales():
+    w = synth.workload(1, scale=0.5)
+    _run_and_compare(make_case(w, no_scales=True), 0)
+    _run_and_compare(make_case(w, pow2_scales=True), 0)
+    case = make_case(w, no_scales=True)
+    case["k_scale"] = None
+    case["v_scale"] = None
+    _run_and_compare(case, 0)
+
+
+def test_stale_out_of_window_table_entries_are_never_read():
+    """Blocks wholly before the window may have been freed: their table entries are junk."""
+    w = synth.Workload("stale", 1, 3, 700, [0], paged=True)
+    case = make_case(w, seq_lens=[700, 400, 129])
+    ref_case = dict(case, table=case["table"].copy())
+    for b, L in enumerate([700, 400, 129]):
+        first_visible_block = (L - 128) // 16
+        case["table"][b, :first_visible_block] = -1
+    dev = _dev(case)
+    dev.append(); oracle_append(ref_case)
+    got, _ = dev.attn(window=128)
+    ref, _ = oracle_attn(ref_case, 128)
+    from gpu_helpers import assert_close
+    assert_close(got, ref, "stale table")
+    assert int(dev.status.item()) == 0
+
+
+def test_device_side_errors_are_flagged_not_faulted():
+    import paper_2602_11937_b200 as P
+    w = synth.Workload("bad", 1, 2, 100, [0], paged=True)
+    case = make_case(w, seq_lens=[100, 100])
+    case["table"][0, 2] = case["num_blocks"] + 5      # out of range
+    case["table"][1, 1] = -3
+    dev = _dev(case)
+    got, _ = dev.attn(window=0)
+    assert int(dev.status.item()) & P.DEV_BAD_BLOCK
+    assert np.isfinite(got).all()                      # the bad blocks read as zeros
+    dev.status.zero_()
+    too_long = torch.tensor([100, 5000], dtype=torch.int32, device="cuda")
+    got, _ = dev.attn(window=0, seq_lens=too_long)
+    assert int(dev.status.item()) & P.DEV_SEQ_TOO_LONG
+
+
+# ------------------------------------------------------------------- merge ---
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_public_merge_matches_oracle(D):
+    import paper_2602_11937_b200 as P
+    rng = np.random.default_rng(11)
+    B, Hq, S = 3, 16, 7
+    po = rng.standard_normal((B, Hq, S, D)).astype(np.float32)
+    pl = (rng.standard_normal((B, Hq, S)) * 4).astype(np.float32)
+    pl[0, :, 2] = -np.inf
+    pl[1, 3, :] = -np.inf
+    po[0, :, 2] = np.nan                       # an empty part's payload must be ignored
+    nparts = np.array([7, 7, 4], dtype=np.int32)
+    sinks = rng.standard_normal(Hq).astype(np.float32)
+    for use_sink in (True, False):
+        out = torch.empty(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty(B, Hq, dtype=torch.float32, device="cuda")
+        P.puzzle_attn_merge(torch.from_numpy(po).cuda(), torch.from_numpy(pl).cuda(), torch.from_numpy(nparts).cuda(),
+                            torch.from_numpy(sinks).cuda() if use_sink else None, out, lse)
+        torch.cuda.synchronize()
+        po_clean = np.nan_to_num(po.astype(np.float64), nan=0.0)
+        ref, ref_lse = oracle.attn_merge(po_clean.reshape(B * Hq, S, D), pl.astype(np.float64).reshape(B * Hq, S),
+                                         np.repeat(nparts, Hq), np.tile(sinks.astype(np.float64), B) if use_sink else None)
+        got = out.float().cpu().numpy().reshape(B * Hq, D)
+        assert np.all(np.abs(got - ref) <= 2e-3 + 2.0 ** -8 * np.abs(ref))
+        gl = lse.cpu().numpy().reshape(-1)
+        fin = np.isfinite(ref_lse)
+        assert np.array_equal(np.isfinite(gl), fin) and np.all(np.abs(gl[fin] - ref_lse[fin]) <= 1e-4)
+
+
+def test_split_partials_are_what_the_oracle_computes_per_split():
+    """The split phase alone: partials of an explicit 2-way split equal the oracle's partial attention."""
+    import paper_2602_11937_b200 as P
+    w = synth.Workload("parts", 1, 1, 256, [0], paged=True)
+    case = make_case(w, seq_lens=[256])
+    dev = _dev(case)
+    dev.append(); oracle_append(case)
+    d = dev.desc(0)
+    nbytes = P.puzzle_decode_attn_workspace_bytes(d, 1, 2)
+    ws = torch.zeros(nbytes // 4, dtype=torch.float32, device="cuda")
+    out = torch.empty(1, 64, 64, dtype=torch.bfloat16, device="cuda")
+    P.puzzle_decode_attn(d, dev.view(), dev.q, None, out, None, num_splits=2, workspace=ws.view(torch.uint8))
+    torch.cuda.synchronize()
+    rows = 64 * 2
+    po = ws[: rows * 64].reshape(64, 2, 64).cpu().numpy().astype(np.float64)
+    pl = ws[rows * 64: rows * 65].reshape(64, 2).cpu().numpy().astype(np.float64)
+    for s, (t0, t1) in enumerate([(0, 128), (128, 256)]):
+        ro, rl = oracle.partial_attn(case["k_cache"], case["v_cache"], 0, case["table"], w.blocks_per_seq,
+                                     case["seq_lens"], case["k_scale"], case["v_scale"], case["q"], case["sm_scale"],
+                                     t0, t1)
+        assert np.all(np.abs(po[:, s] - ro) <= 1e-3)
+        assert np.all(np.abs(pl[:, s] - rl) <= 1e-3)
+
+
+# -------------------------------------------------------------- host errors --
+
+def test_host_side_argument_errors():
+    import paper_2602_11937_b200 as P
+    w = synth.Workload("err", 1, 2, 64, [0], paged=True)
+    dev = _dev(make_case(w))
+    out = torch.empty(2, 64, 64, dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(P.puzzle_decode_attn_workspace_bytes(dev.desc(), 2, 0), dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.PuzzleError) as e:
+        P.puzzle_decode_attn(dev.desc(), dev.view(), dev.q, None, out, None, workspace=ws[:64])
+    assert e.value.code == 4
+    bad = dev.desc()
+    bad.head_dim = 128
+    with pytest.raises(P.PuzzleError) as e:
+        P.puzzle_decode_attn(bad, dev.view(), dev.q, None, out, None, workspace=ws)
+    assert e.value.code == 3
+    bad = dev.desc()
+    bad.num_q_heads = 63
+    with pytest.raises(P.PuzzleError) as e:
+        P.puzzle_decode_attn(bad, dev.view(), dev.q, None, out, None, workspace=ws)
+    assert e.value.code == 2
+    v = dev.view()
+    v.seq_lens = None
+    with pytest.raises(P.PuzzleError) as e:
+        P.puzzle_kv_append(dev.desc(), v, dev.k_new, dev.v_new)
+    assert e.value.code == 1
+    torch.cuda.synchronize()

@@ -1,0 +1,49 @@
+"""CPU-side checks of the boundary: the library loads and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    names = []
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            names += re.findall(r"PUZZLE_API[^;(]*?\b(puzzle_\w+)\s*\(", text)
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2602_11937_b200 import binding, build
+    build.build()
+    lib = ctypes.CDLL(binding.library_path())
+    declared = _declared()
+    assert len(declared) >= 7
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert set(declared) == set(binding.EXPORTS)
+
+
+def test_status_strings_and_workspace_size_need_no_gpu():
+    import paper_2602_11937_b200 as P
+    assert P.puzzle_status_string(0) == "ok"
+    for code in range(1, 6):
+        assert P.puzzle_status_string(code) not in ("ok", "unknown status")
+    d = P.layer_desc()
+    a = P.puzzle_decode_attn_workspace_bytes(d, 16, 0)
+    b = P.puzzle_decode_attn_workspace_bytes(d, 16, 8)
+    assert a > 0 and b == 16 * 64 * 8 * 65 * 4
+    bad = P.layer_desc(head_dim=128)
+    assert P.puzzle_decode_attn_workspace_bytes(bad, 16, 0) == 0
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    from paper_2602_11937_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", "/nonexistent/libpuzzle_attn.so")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.puzzle_launch_count()
