@@ -31,7 +31,7 @@ EncodeTiledFn encode_tiled() {
 
 struct DeviceInfo {
   int sm_count = 0;
-  bool smem_set_fp8 = false;
+  bool smem_attr_set[2] = {false, false};  // per split-KV kernel variant (FP8, bf16)
 };
 DeviceInfo& device_info() {
   static DeviceInfo info[64];
@@ -83,9 +83,13 @@ bool make_cache_map(CUtensorMap* m, void* base, long long rows, int elem_bytes) 
 
 int grid_ctas() { return device_info().sm_count > 0 ? device_info().sm_count : 1; }
 
-size_t workspace_floats(int batch, int Hkv, int num_splits) {
-  const size_t rows = num_splits == 0 ? ((size_t)grid_ctas() * kWarps + (size_t)batch * Hkv) * kGroup
-                                      : (size_t)batch * Hkv * kGroup * num_splits;
+int decode_warps(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kDecodeWarpsFp8 : kDecodeWarpsBf16; }
+int decode_tile(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kTileFp8 : kTileBf16; }
+
+size_t workspace_floats(int batch, int Hkv, int num_splits, int kv_dtype) {
+  const size_t rows = num_splits == 0
+                          ? ((size_t)grid_ctas() * decode_warps(kv_dtype) + (size_t)batch * Hkv) * kGroup
+                          : (size_t)batch * Hkv * kGroup * num_splits;
   return rows * (kHeadDim + 1);
 }
 
@@ -129,7 +133,7 @@ puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_vi
 
 size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits) {
   if (check_desc(desc) != PUZZLE_OK || batch <= 0 || batch > kMaxBatch || num_splits < 0) return 0;
-  return workspace_floats(batch, desc->num_kv_heads, num_splits) * sizeof(float);
+  return workspace_floats(batch, desc->num_kv_heads, num_splits, desc->kv_dtype) * sizeof(float);
 }
 
 puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
@@ -141,9 +145,9 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   if (st != PUZZLE_OK) return st;
   if (!q || !out) return PUZZLE_ERR_NULL;
   if (num_splits < 0 || num_splits > 65536) return PUZZLE_ERR_SHAPE;
-  if (desc->kv_dtype != PUZZLE_KV_FP8_E4M3) return PUZZLE_ERR_UNSUPPORTED;
   const int Hkv = desc->num_kv_heads;
-  const size_t need = workspace_floats(batch, Hkv, num_splits) * sizeof(float);
+  const bool fp8 = desc->kv_dtype == PUZZLE_KV_FP8_E4M3;
+  const size_t need = workspace_floats(batch, Hkv, num_splits, desc->kv_dtype) * sizeof(float);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 15)) return PUZZLE_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 
@@ -155,7 +159,8 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   DecodeParams P;
   std::memset(&P, 0, sizeof P);
   const long long cache_rows = kv->num_blocks * Hkv * (long long)kBlock;
-  if (!make_cache_map(&P.tmK, kv->k_cache, cache_rows, 1) || !make_cache_map(&P.tmV, kv->v_cache, cache_rows, 1))
+  const int eb = fp8 ? 1 : 2;
+  if (!make_cache_map(&P.tmK, kv->k_cache, cache_rows, eb) || !make_cache_map(&P.tmV, kv->v_cache, cache_rows, eb))
     return PUZZLE_ERR_CUDA;
   P.q = static_cast<const __nv_bfloat16*>(q);
   P.block_table = kv->block_table;
@@ -174,17 +179,8 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   P.oob_row = (int)cache_rows;
   P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
 
-  const size_t smem = decode_attn_fp8_smem_bytes(batch);
-  DeviceInfo& di = device_info();
-  if (!di.smem_set_fp8) {
-    if (cudaFuncSetAttribute(decode_attn_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)decode_attn_fp8_smem_bytes(kMaxBatch)) != cudaSuccess)
-      return PUZZLE_ERR_CUDA;
-    di.smem_set_fp8 = true;
-  }
-  decode_attn_fp8_kernel<<<ctas, kWarps * 32, smem, s>>>(P);
+  if (launch_decode_attn(P, fp8, ctas, s, device_info().smem_attr_set) != cudaSuccess) return PUZZLE_ERR_CUDA;
   count_launch();
-  if (cudaGetLastError() != cudaSuccess) return PUZZLE_ERR_CUDA;
 
   MergeParams M;
   std::memset(&M, 0, sizeof M);
@@ -202,7 +198,8 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   M.Hkv = Hkv;
   M.window = desc->window;
   M.max_tokens = kv->max_blocks_per_seq * kBlock;
-  M.num_workers = ctas * kWarps;
+  M.num_workers = ctas * decode_warps(desc->kv_dtype);
+  M.tile = decode_tile(desc->kv_dtype);
   const long long mrows = (long long)batch * desc->num_q_heads;
   attn_merge_kernel<<<(unsigned)((mrows + kWarps - 1) / kWarps), kWarps * 32, attn_merge_smem_bytes(batch, M.balanced),
                       s>>>(M);

@@ -9,7 +9,7 @@ namespace puzzle {
 __global__ void __launch_bounds__(kWarps * 32) attn_merge_kernel(const MergeParams P) {
   extern __shared__ int sched[];  // balanced layout only: cum[batch+1], lens[batch]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (P.balanced) build_schedule(sched, sched + P.batch + 1, P.seq_lens, P.batch, P.Hkv, P.window, P.max_tokens, nullptr);
+  if (P.balanced) build_schedule(sched, sched + P.batch + 1, P.seq_lens, P.batch, P.Hkv, P.window, P.max_tokens, P.tile, nullptr);
 
   const long long row = (long long)blockIdx.x * kWarps + warp;
   if (row >= (long long)P.batch * P.Hq) return;

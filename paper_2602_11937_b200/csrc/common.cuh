@@ -1,6 +1,6 @@
 // Shared device helpers of the decode-attention library: thin wrappers over the
-// sm_100a PTX the kernels use (mbarrier, tiled TMA loads, ldmatrix, FP8 MMA,
-// FP8 conversions).  Header-only; no state.
+// sm_100a PTX the kernels use (mbarrier, tiled TMA loads, ldmatrix, FP8
+// conversions).  Header-only; no state.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -14,8 +14,7 @@ namespace puzzle {
 constexpr int kGroup = 8;     // query heads per KV head
 constexpr int kHeadDim = 64;
 constexpr int kBlock = 16;    // tokens per cache block
-constexpr int kTile = 64;     // tokens one warp consumes per pipeline stage (4 blocks)
-constexpr int kWarps = 8;     // independent workers per CTA
+constexpr int kWarps = 8;     // warps per CTA of the merge kernel (one output row each)
 constexpr int kMaxBatch = 4096;
 
 void count_launch();
@@ -97,40 +96,12 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t& r0, uint3
                : "r"(addr));
 }
 
-// --------------------------------------------------------------------- MMA --
-// D(16x8, f32) += A(16x32, e4m3, row) * B(32x8, e4m3, col)
-__device__ __forceinline__ void mma_e4m3(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
 // ------------------------------------------------------------ conversions --
 // Two floats -> two E4M3 codes (round to nearest even, saturate to +-448);
 // the low byte holds `lo`, the high byte `hi`.
 __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
   uint16_t r;
   asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-// Two E4M3 codes -> two halves (exact).
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t codes) {
-  uint32_t r;
-  uint16_t c = static_cast<uint16_t>(codes);
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(c));
-  return r;
-}
-__device__ __forceinline__ uint32_t f16x2_to_e4m3x2(uint32_t h2) {
-  uint16_t r;
-  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(r) : "r"(h2));
   return r;
 }
 __device__ __forceinline__ uint32_t f32x2_to_f16x2(float lo, float hi) {
@@ -155,30 +126,30 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 }
 
 // ------------------------------------------------- tile schedule (shared) ---
-// Visible key range of a sequence and the 64-token tiles that cover it.
+// Visible key range of a sequence and the tiles (of `tile` tokens) that cover it.
 struct SeqRange {
   int L;     // clamped length
   int lo;    // first visible key
   int tlo;   // first tile
   int ntile; // tiles covering [lo, L)
 };
-__device__ __forceinline__ SeqRange seq_range(int len, int window, int max_tokens, bool& too_long) {
+__device__ __forceinline__ SeqRange seq_range(int len, int window, int max_tokens, int tile, bool& too_long) {
   SeqRange r;
   too_long = len > max_tokens;
   r.L = len < 0 ? 0 : (len > max_tokens ? max_tokens : len);
   r.lo = (window > 0 && r.L > window) ? r.L - window : 0;
-  r.tlo = r.lo / kTile;
-  r.ntile = r.L > 0 ? (r.L + kTile - 1) / kTile - r.tlo : 0;
+  r.tlo = r.lo / tile;
+  r.ntile = r.L > 0 ? (r.L + tile - 1) / tile - r.tlo : 0;
   return r;
 }
 
 // Fills cum[0..batch] (exclusive prefix of ntile * Hkv) and lens[0..batch) in
 // shared memory; every thread of the CTA must call it.  Ends with a CTA barrier.
 __device__ __forceinline__ void build_schedule(int* cum, int* lens, const int32_t* seq_lens, int batch, int Hkv,
-                                               int window, int max_tokens, int32_t* dev_status) {
+                                               int window, int max_tokens, int tile, int32_t* dev_status) {
   for (int b = threadIdx.x; b < batch; b += blockDim.x) {
     bool too_long;
-    SeqRange r = seq_range(seq_lens[b], window, max_tokens, too_long);
+    SeqRange r = seq_range(seq_lens[b], window, max_tokens, tile, too_long);
     if (too_long && dev_status && blockIdx.x == 0) atomicOr(dev_status, (int)PUZZLE_DEV_SEQ_TOO_LONG);
     lens[b] = r.L;
     cum[b + 1] = r.ntile * Hkv;

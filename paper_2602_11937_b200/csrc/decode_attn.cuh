@@ -37,11 +37,17 @@ struct MergeParams {
   // balanced layout: partial rows are addressed as (worker + sequence*Hkv + kv head)*8 + head-in-group
   int balanced;
   const int32_t* seq_lens;
-  int Hkv, window, max_tokens, num_workers;
+  int Hkv, window, max_tokens, num_workers, tile;
 };
 
-__global__ void decode_attn_fp8_kernel(const __grid_constant__ DecodeParams P);
-size_t decode_attn_fp8_smem_bytes(int batch);
+// Shape of the two split-KV kernel variants: warps per CTA (each an independent worker), TMA stages per
+// warp and tokens per tile (the unit of the schedule and of one pipeline stage).
+constexpr int kDecodeWarpsFp8 = 12, kDecodeStagesFp8 = 2, kTileFp8 = 64;
+constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
+
+// Launches the split-KV kernel for an FP8 (fp8 = true) or bf16 cache on `ctas` CTAs.  attr_done[2] caches,
+// per variant, that the dynamic shared-memory limit of the kernel has been raised on the current device.
+cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, bool* attr_done);
 
 __global__ void attn_merge_kernel(const MergeParams P);
 size_t attn_merge_smem_bytes(int batch, int balanced);
