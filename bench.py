@@ -72,7 +72,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
@@ -90,18 +90,18 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
             except Exception:
                 continue
             for n, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w": statistics.median(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
 def physical_gpu_index(local_rank: int) -> int:
@@ -159,6 +159,9 @@ def run_ours(args):
     layers = [build_layer(w, l, dev) for l in range(args.layers)]
     desc = P.layer_desc(window=window, num_q_heads=w.hq, num_kv_heads=w.hkv, head_dim=w.head_dim,
                         block_size=w.block)
+    if args.contiguous:
+        for L in layers:
+            L["table"] = None
     views = [P.kv_view(L["k_cache"], L["v_cache"], seq_lens, block_table=L["table"],
                        max_blocks_per_seq=w.blocks_per_seq, k_scale=L["k_scale"], v_scale=L["v_scale"])
              for L in layers]
@@ -167,6 +170,7 @@ def run_ours(args):
     sinks = synth.draw_sinks(w, 0, dev)
     out = torch.empty(w.batch, w.hq, w.head_dim, dtype=torch.bfloat16, device=dev)
     ws = torch.empty(P.puzzle_decode_attn_workspace_bytes(desc, w.batch, args.splits), dtype=torch.uint8, device=dev)
+    P.puzzle_decode_attn_workspace_init(desc, w.batch, ws)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
@@ -232,6 +236,22 @@ def run_ours(args):
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
+    # ---- read-only streaming probe (one pass over 2 GiB): the bandwidth a pure scan reaches on this device
+    probe_buf = torch.empty(2 << 30, dtype=torch.uint8, device=dev)
+    probe_buf.view(torch.int64).random_()
+    probe_sink = torch.zeros(1, dtype=torch.int64, device=dev)
+    probe_ms = []
+    for i in range(3 + 20):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        P.puzzle_hbm_read_probe(probe_buf, probe_sink, stream=stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        if i >= 3:
+            probe_ms.append(a.elapsed_time(b))
+    probe_gbs = probe_buf.numel() / (statistics.median(probe_ms) * 1e-3) / 1e9
+    del probe_buf
+
     dev_flags = int(status.item())
     bytes_step = algorithmic_bytes(w, seq_lens_host, window)
     kv_bytes_attn = bytes_step - 2 * w.batch * w.hkv * w.head_dim * 3   # what the attention pass itself moves
@@ -251,7 +271,7 @@ def run_ours(args):
             "us_per_layer_step": round(ms_step * 1e3, 2), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp8_e4m3 KV, bf16 q/out, f32 accumulate", "data": "synthetic",
             "config": {"workload": w.name, "batch_per_gpu": w.batch, "context": w.context, "q_heads": w.hq,
-                       "kv_heads": w.hkv, "head_dim": w.head_dim, "block_size": w.block, "window": window,
+                       "kv_heads": w.hkv, "head_dim": w.head_dim, "block_size": w.block, "window": window, "paged": not args.contiguous,
                        "num_splits": args.splits, "rotating_layer_caches": len(layers),
                        "l2": "inputs larger than L2: %.0f MiB per step, %d caches rotated" % (
                            bytes_step / 2 ** 20, len(layers)),
@@ -262,11 +282,12 @@ def run_ours(args):
                     "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in (q, k_new, v_new))),
                     "d2h_bytes_per_step": int(out.numel() * out.element_size())},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "decode_attn_fp8_kernel (+ attn_merge_kernel, same call)",
+            "roofline": {"bound": "hbm", "kernel": "decode_attn_kernel<fp8> (split-KV pass with the merge fused in)",
                          "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
                          "unit": "GB/s", "frac": round(achieved / peak, 4),
                          "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                          "us_per_launch": round(attn_mean_ms * 1e3, 2), "bytes_per_launch": int(kv_bytes_attn),
+                         "read_probe_gbs": round(probe_gbs, 1),
                          "traffic": args.ncu_traffic},
             "dev_status": dev_flags,
         }
@@ -360,6 +381,8 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="workload id 1..5 (3 = batch 16, context 64K)")
     ap.add_argument("--splits", type=int, default=0, help="0 = balanced schedule, S = fixed splits per sequence")
     ap.add_argument("--layers", type=int, default=4, help="distinct layer caches rotated between steps")
+    ap.add_argument("--contiguous", action="store_true",
+                    help="diagnostic: drop the block table (sequence b owns blocks b*blocks_per_seq ...)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--ncu-traffic", type=float, default=None,
                     help="DRAM bytes per launch of the attention kernel from an ncu capture (reported as-is)")

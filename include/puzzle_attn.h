@@ -104,6 +104,17 @@ PUZZLE_API puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const p
  * (0 on invalid arguments).  num_splits == 0 selects the balanced schedule. */
 PUZZLE_API size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits);
 
+/* Prepares a freshly allocated workspace: zero-fills the arrival counters at
+ * its start (one int32 per (sequence, KV head), padded to 256 bytes) on
+ * `stream`.  Call it once per workspace before its first puzzle_decode_attn;
+ * every completed puzzle_decode_attn leaves the counters at zero again, for any
+ * batch and split choice that fits the workspace.  Call it again after a step
+ * whose *dev_status reported PUZZLE_DEV_WAIT_EXPIRED (that step stopped half
+ * way).  The split-KV phase of Section "Optimized Scenarios"' KV-bound decode
+ * needs these counters to know which worker finishes a (sequence, KV head). */
+PUZZLE_API puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_desc* desc, int32_t batch,
+                                                           void* workspace, size_t workspace_bytes, void* stream);
+
 /* Decode-step attention of one layer: for every sequence b and query head g
  * (KV head h = g / 8), over the visible keys j in [L - min(W, L), L) with
  * L = seq_lens[b] (all of [0, L) when window == 0):
@@ -111,14 +122,16 @@ PUZZLE_API size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* de
  *     Z = e^(sink_g - M) + sum_j e^(s_j - M),  out = v_scale[h] * sum_j e^(s_j - M) Vcode_j / Z.
  * Full vs window is the paper's per-layer choice (Section "Window attention for
  * long-context inference"); the sink is one extra softmax column per query head
- * that carries no value.  Internally: a split-KV pass that writes float32
- * partial (o, lse) into the workspace, then a log-sum-exp merge.
- *   q: bf16 [batch][num_q_heads][head_dim];  sinks: float32 [num_q_heads] or NULL (no sink);
- *   out: bf16 [batch][num_q_heads][head_dim];  lse_out: float32 [batch][num_q_heads] or NULL;
+ * that carries no value.  Internally ONE kernel: a split-KV pass writes float32
+ * partial (o, lse) into the workspace, and the worker that completes a
+ * (sequence, KV head) merges its partials by log-sum-exp and writes `out`.
+ *   q: bf16 [batch][num_q_heads][head_dim], 8-byte aligned;  sinks: float32 [num_q_heads] or NULL (no sink);
+ *   out: bf16 [batch][num_q_heads][head_dim], 16-byte aligned;  lse_out: float32 [batch][num_q_heads] or NULL;
  *   num_splits: 0 = balanced schedule (recommended); S >= 1 = every (sequence, KV head) context is
  *     cut into S equal runs of 64-token tiles;
  *   workspace: device scratch of at least puzzle_decode_attn_workspace_bytes(...) bytes, 16-byte
- *     aligned, contents undefined before and after;
+ *     aligned, prepared once by puzzle_decode_attn_workspace_init; calls that share a workspace must
+ *     not overlap on the GPU;
  *   dev_status: optional int32 device word (see PUZZLE_DEV_*).
  * An empty context gives out = 0 and lse = sink (-inf without a sink). */
 PUZZLE_API puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
@@ -126,9 +139,9 @@ PUZZLE_API puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const
                                  int32_t num_splits, void* workspace, size_t workspace_bytes,
                                  int32_t* dev_status, void* stream);
 
-/* Log-sum-exp merge of partial attention results (the second phase above, also
- * usable on partials that came from elsewhere, e.g. context shards on other
- * GPUs).  For every row r = (b, g):
+/* Log-sum-exp merge of partial attention results that came from elsewhere
+ * (e.g. context shards on other GPUs; puzzle_decode_attn merges its own
+ * partials itself).  For every row r = (b, g):
  *     M = max(sink_g, max_p lse_p),  Z = e^(sink_g - M) + sum_p e^(lse_p - M),
  *     out = sum_p e^(lse_p - M) o_p / Z,  lse_out = M + ln Z.
  *   part_o: float32 [batch][Hq][S][D];  part_lse: float32 [batch][Hq][S] (natural log; -inf = empty part);

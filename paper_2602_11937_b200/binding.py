@@ -8,7 +8,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "lib", "libpuzzle_attn.so")
+# PUZZLE_ATTN_LIB points the binding at another build of the same library (e.g. a tuning variant)
+_LIB_PATH = os.environ.get("PUZZLE_ATTN_LIB") or os.path.join(_HERE, "lib", "libpuzzle_attn.so")
 _lib = None
 
 KV_FP8_E4M3 = 0
@@ -20,6 +21,7 @@ DEV_WAIT_EXPIRED = 4
 EXPORTS = (
     "puzzle_kv_append",
     "puzzle_decode_attn_workspace_bytes",
+    "puzzle_decode_attn_workspace_init",
     "puzzle_decode_attn",
     "puzzle_attn_merge",
     "puzzle_hbm_read_probe",
@@ -63,6 +65,8 @@ def _load():
         lib.puzzle_kv_append.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, i32, vp, vp]
         lib.puzzle_decode_attn_workspace_bytes.restype = sz
         lib.puzzle_decode_attn_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32, i32]
+        lib.puzzle_decode_attn_workspace_init.restype = ctypes.c_int
+        lib.puzzle_decode_attn_workspace_init.argtypes = [ctypes.POINTER(LayerDesc), i32, vp, sz, vp]
         lib.puzzle_decode_attn.restype = ctypes.c_int
         lib.puzzle_decode_attn.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp, i32, i32,
                                            vp, sz, vp, vp]
@@ -148,6 +152,12 @@ def puzzle_kv_append(desc: LayerDesc, view: KVView, k_new: torch.Tensor, v_new: 
 
 def puzzle_decode_attn_workspace_bytes(desc: LayerDesc, batch: int, num_splits: int = 0) -> int:
     return int(_load().puzzle_decode_attn_workspace_bytes(ctypes.byref(desc), int(batch), int(num_splits)))
+
+
+def puzzle_decode_attn_workspace_init(desc: LayerDesc, batch: int, workspace: torch.Tensor, stream=None) -> None:
+    _check(_load().puzzle_decode_attn_workspace_init(ctypes.byref(desc), int(batch), _p(workspace),
+                                                     workspace.numel() * workspace.element_size(), _stream(stream)),
+           "puzzle_decode_attn_workspace_init")
 
 
 def puzzle_decode_attn(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Optional[torch.Tensor],

@@ -31,7 +31,7 @@ EncodeTiledFn encode_tiled() {
 
 struct DeviceInfo {
   int sm_count = 0;
-  bool smem_attr_set[2] = {false, false};  // per split-KV kernel variant (FP8, bf16)
+  int smem_limit[2] = {0, 0};  // per split-KV kernel variant (FP8, bf16); 0 = not raised yet
 };
 DeviceInfo& device_info() {
   static DeviceInfo info[64];
@@ -86,6 +86,9 @@ int grid_ctas() { return device_info().sm_count > 0 ? device_info().sm_count : 1
 int decode_warps(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kDecodeWarpsFp8 : kDecodeWarpsBf16; }
 int decode_tile(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kTileFp8 : kTileBf16; }
 
+// The workspace starts with one arrival counter per (sequence, KV head), padded to 256 bytes.
+size_t counter_bytes(int batch, int Hkv) { return (((size_t)batch * Hkv * sizeof(int32_t)) + 255) & ~(size_t)255; }
+
 size_t workspace_floats(int batch, int Hkv, int num_splits, int kv_dtype) {
   const size_t rows = num_splits == 0
                           ? ((size_t)grid_ctas() * decode_warps(kv_dtype) + (size_t)batch * Hkv) * kGroup
@@ -133,7 +136,8 @@ puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_vi
 
 size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits) {
   if (check_desc(desc) != PUZZLE_OK || batch <= 0 || batch > kMaxBatch || num_splits < 0) return 0;
-  return workspace_floats(batch, desc->num_kv_heads, num_splits, desc->kv_dtype) * sizeof(float);
+  return counter_bytes(batch, desc->num_kv_heads) +
+         workspace_floats(batch, desc->num_kv_heads, num_splits, desc->kv_dtype) * sizeof(float);
 }
 
 puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
@@ -145,15 +149,18 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   if (st != PUZZLE_OK) return st;
   if (!q || !out) return PUZZLE_ERR_NULL;
   if (num_splits < 0 || num_splits > 65536) return PUZZLE_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(q) & 7) || (reinterpret_cast<uintptr_t>(out) & 15)) return PUZZLE_ERR_SHAPE;
   const int Hkv = desc->num_kv_heads;
   const bool fp8 = desc->kv_dtype == PUZZLE_KV_FP8_E4M3;
-  const size_t need = workspace_floats(batch, Hkv, num_splits, desc->kv_dtype) * sizeof(float);
+  const size_t cbytes = counter_bytes(batch, Hkv);
+  const size_t pfloats = workspace_floats(batch, Hkv, num_splits, desc->kv_dtype);
+  const size_t need = cbytes + pfloats * sizeof(float);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 15)) return PUZZLE_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 
   const int ctas = grid_ctas();
-  const size_t rows = need / sizeof(float) / (kHeadDim + 1);
-  float* part_o = static_cast<float*>(workspace);
+  const size_t rows = pfloats / (kHeadDim + 1);
+  float* part_o = reinterpret_cast<float*>(static_cast<char*>(workspace) + cbytes);
   float* part_lse = part_o + rows * kHeadDim;
 
   DecodeParams P;
@@ -169,6 +176,10 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   P.v_scale = kv->v_scale;
   P.part_o = part_o;
   P.part_lse = part_lse;
+  P.counters = static_cast<int32_t*>(workspace);
+  P.sinks = sinks;
+  P.out = static_cast<__nv_bfloat16*>(out);
+  P.lse_out = lse_out;
   P.dev_status = dev_status;
   P.num_blocks = kv->num_blocks;
   P.batch = batch;
@@ -179,32 +190,22 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   P.oob_row = (int)cache_rows;
   P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
 
-  if (launch_decode_attn(P, fp8, ctas, s, device_info().smem_attr_set) != cudaSuccess) return PUZZLE_ERR_CUDA;
+  if (launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit) != cudaSuccess) return PUZZLE_ERR_CUDA;
   count_launch();
 
-  MergeParams M;
-  std::memset(&M, 0, sizeof M);
-  M.part_o = part_o;
-  M.part_lse = part_lse;
-  M.sinks = sinks;
-  M.out = static_cast<__nv_bfloat16*>(out);
-  M.lse_out = lse_out;
-  M.batch = batch;
-  M.Hq = desc->num_q_heads;
-  M.D = kHeadDim;
-  M.S = num_splits;
-  M.balanced = num_splits == 0;
-  M.seq_lens = kv->seq_lens;
-  M.Hkv = Hkv;
-  M.window = desc->window;
-  M.max_tokens = kv->max_blocks_per_seq * kBlock;
-  M.num_workers = ctas * decode_warps(desc->kv_dtype);
-  M.tile = decode_tile(desc->kv_dtype);
-  const long long mrows = (long long)batch * desc->num_q_heads;
-  attn_merge_kernel<<<(unsigned)((mrows + kWarps - 1) / kWarps), kWarps * 32, attn_merge_smem_bytes(batch, M.balanced),
-                      s>>>(M);
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+  return PUZZLE_OK;
+}
+
+puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_desc* desc, int32_t batch, void* workspace,
+                                                size_t workspace_bytes, void* stream) {
+  puzzle_status st = check_desc(desc);
+  if (st != PUZZLE_OK) return st;
+  if (batch <= 0 || batch > kMaxBatch) return PUZZLE_ERR_SHAPE;
+  const size_t cbytes = counter_bytes(batch, desc->num_kv_heads);
+  if (!workspace || workspace_bytes < cbytes || (reinterpret_cast<uintptr_t>(workspace) & 15))
+    return PUZZLE_ERR_WORKSPACE;
+  return cudaMemsetAsync(workspace, 0, cbytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PUZZLE_OK
+                                                                                                  : PUZZLE_ERR_CUDA;
 }
 
 puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, const int32_t* num_parts,
@@ -226,7 +227,6 @@ puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, cons
   M.Hq = Hq;
   M.D = D;
   M.S = S;
-  M.balanced = 0;
   const long long rows = (long long)batch * Hq;
   attn_merge_kernel<<<(unsigned)((rows + kWarps - 1) / kWarps), kWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(M);
   count_launch();

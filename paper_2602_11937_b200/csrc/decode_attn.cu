@@ -27,7 +27,9 @@
 //  * Work is cut into tiles; in the balanced schedule the tile space of the
 //    whole batch is divided evenly over all workers (ragged contexts and window
 //    layers included), each worker writing one float32 partial (o, lse) per
-//    (sequence, KV head) run it touches.  A merge kernel combines them.
+//    (sequence, KV head) run it touches.  The worker whose partial completes a
+//    (sequence, KV head) merges all of them (log-sum-exp, sink folded in once)
+//    and writes the bf16 output: one launch per layer, no waiting anywhere.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -184,6 +186,101 @@ __device__ __forceinline__ void mma_bf16v(float (&c)[4], uint32_t a0, uint32_t a
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+
+// Log-sum-exp merge of the `count` partials of one (sequence, KV head) by one warp: the quad of lanes with
+// g = lane/4 owns query head g of the group, lane c = lane%4 of the quad owns channels 16c..16c+15.
+//   M = max(sink, max_k lse_k);  Z = e^(sink-M) + sum_k e^(lse_k-M);  out = sum_k e^(lse_k-M) o_k / Z.
+// Part k of head g is partial row first + g*hstride + k*kstride.  The partials were written by other SMs
+// in this launch, so they are read past L1.
+__device__ __forceinline__ void merge_rows(const DecodeParams& P, int b, int kvh, long long first, int count,
+                                           int kstride, int hstride, int lane) {
+  const int g = lane >> 2, c = lane & 3;
+  const int Hq = P.Hkv * kGroup, head = kvh * kGroup + g;
+  const long long row_out = (long long)b * Hq + head;
+  const float sink = P.sinks ? P.sinks[head] : -INFINITY;
+  const long long base = first + (long long)g * hstride;
+  float M = -INFINITY;
+  for (int k = c; k < count; k += 4) M = fmaxf(M, __ldcg(P.part_lse + base + (long long)k * kstride));
+  M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
+  M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
+  M = fmaxf(M, sink);
+  float acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+  float Z = 0.f;
+  if (M != -INFINITY) {
+    // four parts per round, every load of the round issued before the first use: the merge is a chain of
+    // L2 round trips, so their number, not the arithmetic, sets its duration
+    for (int k0 = 0; k0 < count; k0 += 4) {
+      float l[4];
+      float4 v[4][4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool on = k0 + j < count;
+        const long long idx = base + (long long)(on ? k0 + j : k0) * kstride;
+        l[j] = on ? __ldcg(P.part_lse + idx) : -INFINITY;
+        const float4* o = reinterpret_cast<const float4*>(P.part_o + idx * kHeadDim + 16 * c);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[j][i] = __ldcg(o + i);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (l[j] == -INFINITY) continue;  // an empty part: its payload is undefined
+        const float wgt = __expf(l[j] - M);
+        Z += wgt;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[4 * i + 0] += wgt * v[j][i].x; acc[4 * i + 1] += wgt * v[j][i].y;
+          acc[4 * i + 2] += wgt * v[j][i].z; acc[4 * i + 3] += wgt * v[j][i].w;
+        }
+      }
+    }
+    if (sink != -INFINITY) Z += __expf(sink - M);  // the sink is one more softmax column, counted once
+  }
+  const float invZ = Z > 0.f ? 1.f / Z : 0.f;  // nothing visible and no sink: zeros
+  uint32_t packed[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) packed[i] = f32x2_to_bf16x2(acc[2 * i] * invZ, acc[2 * i + 1] * invZ);
+  uint4* dst = reinterpret_cast<uint4*>(P.out + row_out * kHeadDim + 16 * c);
+  dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+  dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+  if (P.lse_out && c == 0) P.lse_out[row_out] = Z > 0.f ? M + __logf(Z) : -INFINITY;
+}
+
+// Called by a warp after it has stored its partial of (sequence b, KV head kvh): counts the arrival, and the
+// warp that completes the set merges it and leaves the counter at zero for the next launch.
+__device__ __forceinline__ void arrive_and_merge(const DecodeParams& P, int b, int kvh, const int* cum, int nW,
+                                                 int lane) {
+  const int p = b * P.Hkv + kvh;
+  long long first;
+  int count, kstride, hstride;
+  if (P.num_splits == 0) {
+    const int nt = (cum[b + 1] - cum[b]) / P.Hkv;
+    const int T = cum[P.batch];
+    const int q = (T + nW - 1) / nW;
+    const int g0 = cum[b] + kvh * nt;
+    const int w0 = g0 / q, w1 = (g0 + nt - 1) / q;
+    first = ((long long)w0 + p) * kGroup;
+    count = w1 - w0 + 1;
+    kstride = kGroup;
+    hstride = 1;
+  } else {
+    first = (long long)p * kGroup * P.num_splits;
+    count = P.num_splits;
+    kstride = 1;
+    hstride = P.num_splits;
+  }
+  __threadfence();  // this lane's partial stores before the arrival
+  __syncwarp();
+  int last = 0;
+  if (lane == 0) last = atomicAdd(P.counters + p, 1) == count - 1;
+  last = __shfl_sync(0xffffffffu, last, 0);
+  if (!last) return;
+  __threadfence();  // the arrivals before the other warps' partials are read
+  merge_rows(P, b, kvh, first, count, kstride, hstride, lane);
+  if (lane == 0) P.counters[p] = 0;
+}
+
 }  // namespace
 
 // NW warps per CTA, NS stages per warp, TT tokens per tile; FP8 selects the E4M3 cache (else bf16).
@@ -276,6 +373,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
   while (!failed && next_segment<TT>(cc, cs, P, cum, lens, w)) {
     if (cs.t == cs.t_end) {  // empty split: weight zero
       if (c == 0) P.part_lse[cs.prow + g * cs.pstride] = -INFINITY;
+      arrive_and_merge(P, cs.b, cs.kvh, cum, nW, lane);
       continue;
     }
     // ---- query of this (sequence, KV head) as A-fragments (rows 0-7 = heads, rows 8-15 unused)
@@ -497,6 +595,15 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     for (int nd = 0; nd < 8; ++nd)
       *reinterpret_cast<float2*>(po + 8 * nd) = make_float2((O[nd][0] + O[nd][2]) * inv, (O[nd][1] + O[nd][3]) * inv);
     if (c == 0) P.part_lse[row] = lse;
+    arrive_and_merge(P, cs.b, cs.kvh, cum, nW, lane);
+  }
+
+  // sequences without any visible key have no tile and hence no worker in the balanced schedule
+  if (!failed && P.num_splits == 0) {
+    for (int p = w; p < P.batch * P.Hkv; p += nW) {
+      const int b = p / P.Hkv;
+      if (cum[b + 1] == cum[b]) merge_rows(P, b, p - b * P.Hkv, 0, 0, 0, 0, lane);
+    }
   }
 
   if (failed) {
@@ -515,21 +622,25 @@ static size_t smem_bytes_of(int batch) {
 }
 
 template <int NW, int NS, int TT, bool FP8>
-static cudaError_t launch_variant(const DecodeParams& P, int ctas, cudaStream_t s, bool& attr_done) {
+static cudaError_t launch_variant(const DecodeParams& P, int ctas, cudaStream_t s, int& smem_limit) {
   auto kern = decode_attn_kernel<NW, NS, TT, FP8>;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem_bytes_of<NW, NS, TT, FP8>(kMaxBatch));
+  if (smem_limit == 0) {  // first launch of this variant on this device: raise its dynamic shared-memory limit
+    int dev = 0, optin = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, optin);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    smem_limit = optin;
   }
-  kern<<<ctas, NW * 32, smem_bytes_of<NW, NS, TT, FP8>(P.batch), s>>>(P);
+  const size_t need = smem_bytes_of<NW, NS, TT, FP8>(P.batch);
+  if (need > (size_t)smem_limit) return cudaErrorInvalidValue;  // batch too large for the schedule arrays
+  kern<<<ctas, NW * 32, need, s>>>(P);
   return cudaGetLastError();
 }
 
-cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, bool* attr_done) {
-  return fp8 ? launch_variant<kDecodeWarpsFp8, kDecodeStagesFp8, kTileFp8, true>(P, ctas, s, attr_done[0])
-             : launch_variant<kDecodeWarpsBf16, kDecodeStagesBf16, kTileBf16, false>(P, ctas, s, attr_done[1]);
+cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit) {
+  return fp8 ? launch_variant<kDecodeWarpsFp8, kDecodeStagesFp8, kTileFp8, true>(P, ctas, s, smem_limit[0])
+             : launch_variant<kDecodeWarpsBf16, kDecodeStagesBf16, kTileBf16, false>(P, ctas, s, smem_limit[1]);
 }
 
 }  // namespace puzzle

@@ -18,6 +18,10 @@ struct alignas(64) DecodeParams {
   const float* v_scale;
   float* part_o;
   float* part_lse;
+  int32_t* counters;   // [batch*Hkv] arrivals per (sequence, KV head); zero before and after every launch
+  const float* sinks;  // [Hq] or null
+  __nv_bfloat16* out;  // [batch][Hq][D]
+  float* lse_out;      // [batch][Hq] or null
   int32_t* dev_status;
   long long num_blocks;
   int batch, Hkv, max_blocks_per_seq, window;
@@ -27,30 +31,30 @@ struct alignas(64) DecodeParams {
 };
 
 struct MergeParams {
-  const float* part_o;
-  const float* part_lse;
-  const int32_t* num_parts;  // explicit layout only
+  const float* part_o;       // [rows][S][D]
+  const float* part_lse;     // [rows][S]
+  const int32_t* num_parts;  // [batch] or null
   const float* sinks;
   __nv_bfloat16* out;
   float* lse_out;
   int batch, Hq, D, S;
-  // balanced layout: partial rows are addressed as (worker + sequence*Hkv + kv head)*8 + head-in-group
-  int balanced;
-  const int32_t* seq_lens;
-  int Hkv, window, max_tokens, num_workers, tile;
 };
 
 // Shape of the two split-KV kernel variants: warps per CTA (each an independent worker), TMA stages per
 // warp and tokens per tile (the unit of the schedule and of one pipeline stage).
-constexpr int kDecodeWarpsFp8 = 12, kDecodeStagesFp8 = 2, kTileFp8 = 64;
+#ifndef PUZZLE_FP8_WARPS
+#define PUZZLE_FP8_WARPS 12
+#define PUZZLE_FP8_STAGES 2
+#define PUZZLE_FP8_TILE 64
+#endif
+constexpr int kDecodeWarpsFp8 = PUZZLE_FP8_WARPS, kDecodeStagesFp8 = PUZZLE_FP8_STAGES, kTileFp8 = PUZZLE_FP8_TILE;
 constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
 
-// Launches the split-KV kernel for an FP8 (fp8 = true) or bf16 cache on `ctas` CTAs.  attr_done[2] caches,
-// per variant, that the dynamic shared-memory limit of the kernel has been raised on the current device.
-cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, bool* attr_done);
+// Launches the split-KV kernel for an FP8 (fp8 = true) or bf16 cache on `ctas` CTAs.  smem_limit[2] caches,
+// per variant, the dynamic shared-memory limit set for the kernel on the current device (0 = not set yet).
+cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit);
 
 __global__ void attn_merge_kernel(const MergeParams P);
-size_t attn_merge_smem_bytes(int batch, int balanced);
 
 __global__ void kv_append_kernel(void* k_cache, void* v_cache, const __nv_bfloat16* k_new,
                                  const __nv_bfloat16* v_new, const int32_t* block_table, const int32_t* seq_lens,

@@ -59,6 +59,7 @@ class DeviceCase:
         ws = torch.empty(max(16, P.puzzle_decode_attn_workspace_bytes(d, w.batch, num_splits)), dtype=torch.uint8,
                          device="cuda")
         ws.fill_(0xFF)  # NaN patterns: stale scratch must never leak into results
+        P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
         out = torch.full((w.batch, w.hq, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
         lse = torch.full((w.batch, w.hq), float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
         s = self.sinks if isinstance(sinks, str) else sinks

@@ -257,8 +257,10 @@ def test_split_partials_are_what_the_oracle_computes_per_split():
     P.puzzle_decode_attn(d, dev.view(), dev.q, None, out, None, num_splits=2, workspace=ws.view(torch.uint8))
     torch.cuda.synchronize()
     rows = 64 * 2
-    po = ws[: rows * 64].reshape(64, 2, 64).cpu().numpy().astype(np.float64)
-    pl = ws[rows * 64: rows * 65].reshape(64, 2).cpu().numpy().astype(np.float64)
+    part = ws[256 // 4:]                       # the partials follow the 256-byte counter block
+    assert not ws[: 256 // 4].any()            # which a finished call leaves at zero
+    po = part[: rows * 64].reshape(64, 2, 64).cpu().numpy().astype(np.float64)
+    pl = part[rows * 64: rows * 65].reshape(64, 2).cpu().numpy().astype(np.float64)
     for s, (t0, t1) in enumerate([(0, 128), (128, 256)]):
         ro, rl = oracle.partial_attn(case["k_cache"], case["v_cache"], 0, case["table"], w.blocks_per_seq,
                                      case["seq_lens"], case["k_scale"], case["v_scale"], case["q"], case["sm_scale"],
@@ -274,7 +276,7 @@ def test_host_side_argument_errors():
     w = synth.Workload("err", 1, 2, 64, [0], paged=True)
     dev = _dev(make_case(w))
     out = torch.empty(2, 64, 64, dtype=torch.bfloat16, device="cuda")
-    ws = torch.empty(P.puzzle_decode_attn_workspace_bytes(dev.desc(), 2, 0), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(dev.desc(), 2, 0), dtype=torch.uint8, device="cuda")
     with pytest.raises(P.PuzzleError) as e:
         P.puzzle_decode_attn(dev.desc(), dev.view(), dev.q, None, out, None, workspace=ws[:64])
     assert e.value.code == 4
