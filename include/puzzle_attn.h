@@ -139,6 +139,35 @@ PUZZLE_API puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const
                                  int32_t num_splits, void* workspace, size_t workspace_bytes,
                                  int32_t* dev_status, void* stream);
 
+/* Size of the scratch array built into the library for puzzle_decode_attn_static. */
+#define PUZZLE_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* puzzle_decode_attn without a workspace argument, for callers that cannot
+ * allocate device memory where they call it: a server that gave all free HBM to
+ * its KV-cache pool at start-up, code hosted inside another runtime whose
+ * allocator it must not use, or a decode loop whose rules forbid cudaMalloc
+ * because it stalls the whole device.  (The paper has no counterpart; this is a
+ * deployment convenience.)  Results are those of puzzle_decode_attn, argument
+ * for argument; inputs and outputs are still the caller's.
+ *   - The scratch is a fixed PUZZLE_STATIC_SCRATCH_BYTES (8 MiB) array inside
+ *     the library's device image; every GPU that loads the library holds it until
+ *     the process exits.  A batch and split choice whose
+ *     puzzle_decode_attn_workspace_bytes exceeds that size is refused with
+ *     PUZZLE_ERR_WORKSPACE and nothing is launched (balanced schedule: batch up
+ *     to about 280; explicit splits: batch * num_splits up to about 500).
+ *   - The call allocates and frees nothing.  The first call on each device looks
+ *     up the array's device address (with that device current); make that first
+ *     call before starting any stream capture.
+ *   - All calls on a device share the one array.  Two calls that overlap on the
+ *     GPU (different streams, no dependency between them) race on it and both
+ *     results are undefined; order them.  The array keeps the previous call's
+ *     contents; the part that must start at zero is cleared on `stream` by every
+ *     call before its kernel. */
+PUZZLE_API puzzle_status puzzle_decode_attn_static(const puzzle_layer_desc* desc, const puzzle_kv_view* kv,
+                                                   const void* q, const float* sinks, void* out, float* lse_out,
+                                                   int32_t batch, int32_t num_splits, int32_t* dev_status,
+                                                   void* stream);
+
 /* Log-sum-exp merge of partial attention results that came from elsewhere
  * (e.g. context shards on other GPUs; puzzle_decode_attn merges its own
  * partials itself).  For every row r = (b, g):

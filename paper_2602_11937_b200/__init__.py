@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     DEV_BAD_BLOCK,
     DEV_SEQ_TOO_LONG,
     DEV_WAIT_EXPIRED,
+    STATIC_SCRATCH_BYTES,
     KVView,
     LayerDesc,
     PuzzleError,
@@ -18,6 +19,7 @@ from .binding import (  # noqa: F401
     library_path,
     puzzle_attn_merge,
     puzzle_decode_attn,
+    puzzle_decode_attn_static,
     puzzle_decode_attn_workspace_bytes,
     puzzle_decode_attn_workspace_init,
     puzzle_hbm_read_probe,

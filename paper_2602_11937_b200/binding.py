@@ -17,12 +17,14 @@ KV_BF16 = 1
 DEV_BAD_BLOCK = 1
 DEV_SEQ_TOO_LONG = 2
 DEV_WAIT_EXPIRED = 4
+STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = (
     "puzzle_kv_append",
     "puzzle_decode_attn_workspace_bytes",
     "puzzle_decode_attn_workspace_init",
     "puzzle_decode_attn",
+    "puzzle_decode_attn_static",
     "puzzle_attn_merge",
     "puzzle_hbm_read_probe",
     "puzzle_status_string",
@@ -70,6 +72,9 @@ def _load():
         lib.puzzle_decode_attn.restype = ctypes.c_int
         lib.puzzle_decode_attn.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp, i32, i32,
                                            vp, sz, vp, vp]
+        lib.puzzle_decode_attn_static.restype = ctypes.c_int
+        lib.puzzle_decode_attn_static.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp,
+                                                  i32, i32, vp, vp]
         lib.puzzle_attn_merge.restype = ctypes.c_int
         lib.puzzle_attn_merge.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
         lib.puzzle_hbm_read_probe.restype = ctypes.c_int
@@ -172,6 +177,19 @@ def puzzle_decode_attn(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Op
                                       _p(lse_out, torch.float32, "lse_out"), batch, int(num_splits), _p(workspace),
                                       workspace.numel() * workspace.element_size(), _p(dev_status, torch.int32),
                                       _stream(stream)), "puzzle_decode_attn")
+
+
+def puzzle_decode_attn_static(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Optional[torch.Tensor],
+                              out: torch.Tensor, lse_out: Optional[torch.Tensor] = None, num_splits: int = 0,
+                              dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """puzzle_decode_attn on the library's built-in 8 MiB scratch: for callers that cannot allocate device
+    memory (no workspace tensor is involved, and nothing is allocated on the way).  Calls that share a
+    device must not overlap on the GPU; make the first call on a device outside any stream capture."""
+    _check(_load().puzzle_decode_attn_static(ctypes.byref(desc), ctypes.byref(view), _p(q, torch.bfloat16, "q"),
+                                             _p(sinks, torch.float32, "sinks"), _p(out, torch.bfloat16, "out"),
+                                             _p(lse_out, torch.float32, "lse_out"), q.shape[0], int(num_splits),
+                                             _p(dev_status, torch.int32), _stream(stream)),
+           "puzzle_decode_attn_static")
 
 
 def puzzle_attn_merge(part_o: torch.Tensor, part_lse: torch.Tensor, num_parts: Optional[torch.Tensor],

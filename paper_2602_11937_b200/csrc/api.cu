@@ -84,7 +84,6 @@ bool make_cache_map(CUtensorMap* m, void* base, long long rows, int elem_bytes) 
 int grid_ctas() { return device_info().sm_count > 0 ? device_info().sm_count : 1; }
 
 int decode_warps(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kDecodeWarpsFp8 : kDecodeWarpsBf16; }
-int decode_tile(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kTileFp8 : kTileBf16; }
 
 // The workspace starts with one arrival counter per (sequence, KV head), padded to 256 bytes.
 size_t counter_bytes(int batch, int Hkv) { return (((size_t)batch * Hkv * sizeof(int32_t)) + 255) & ~(size_t)255; }
