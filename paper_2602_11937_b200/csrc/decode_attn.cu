@@ -192,7 +192,7 @@ __device__ __forceinline__ void mma_bf16v(float (&c)[4], uint32_t a0, uint32_t a
 //   M = max(sink, max_k lse_k);  Z = e^(sink-M) + sum_k e^(lse_k-M);  out = sum_k e^(lse_k-M) o_k / Z.
 // Part k of head g is partial row first + g*hstride + k*kstride.  The partials were written by other SMs
 // in this launch, so they are read past L1.
-__device__ __forceinline__ void merge_rows(const DecodeParams& P, int b, int kvh, long long first, int count,
+__device__ __noinline__ void merge_rows(const DecodeParams& P, int b, int kvh, long long first, int count,
                                            int kstride, int hstride, int lane) {
   const int g = lane >> 2, c = lane & 3;
   const int Hq = P.Hkv * kGroup, head = kvh * kGroup + g;
