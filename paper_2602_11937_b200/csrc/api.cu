@@ -65,18 +65,18 @@ puzzle_status check_view(const puzzle_layer_desc* d, const puzzle_kv_view* kv, i
   return PUZZLE_OK;
 }
 
-// 2-D view of a cache: rows = (block, kv head, slot), one row = one token's head_dim elements.
-// Box = one 16-token block of one KV head; swizzle spans one row (64 B for FP8, 128 B for bf16).
+// 2-D view of a cache as rows of 128 bytes: two FP8 tokens or one bf16 token per row, so that every TMA
+// request is a full 128-byte line.  Box = one 16-token block of one KV head (8 or 16 rows), 128-byte swizzle.
 bool make_cache_map(CUtensorMap* m, void* base, long long rows, int elem_bytes) {
   EncodeTiledFn enc = encode_tiled();
   if (!enc) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * elem_bytes};
-  const cuuint32_t box[2] = {(cuuint32_t)kHeadDim, (cuuint32_t)kBlock};
+  const cuuint64_t inner = 128 / elem_bytes;  // elements per row
+  const cuuint64_t dims[2] = {inner, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {(cuuint32_t)inner, (cuuint32_t)(kBlock * kHeadDim * elem_bytes / 128)};
   const cuuint32_t estr[2] = {1, 1};
   CUresult r = enc(m, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base,
-                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   elem_bytes == 1 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -164,8 +164,9 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
 
   DecodeParams P;
   std::memset(&P, 0, sizeof P);
-  const long long cache_rows = kv->num_blocks * Hkv * (long long)kBlock;
   const int eb = fp8 ? 1 : 2;
+  const int rows_per_block = kBlock * kHeadDim * eb / 128;
+  const long long cache_rows = kv->num_blocks * Hkv * (long long)rows_per_block;
   if (!make_cache_map(&P.tmK, kv->k_cache, cache_rows, eb) || !make_cache_map(&P.tmV, kv->v_cache, cache_rows, eb))
     return PUZZLE_ERR_CUDA;
   P.q = static_cast<const __nv_bfloat16*>(q);
@@ -187,6 +188,7 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   P.window = desc->window;
   P.num_splits = num_splits;
   P.oob_row = (int)cache_rows;
+  P.rows_per_block = rows_per_block;
   P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
 
   if (launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit) != cudaSuccess) return PUZZLE_ERR_CUDA;

@@ -139,7 +139,7 @@ struct Producer {
     if (lane < 2 * NB) {
       int row = P.oob_row;
       if (phys >= 0 && phys < P.num_blocks) {
-        row = (int)((phys * P.Hkv + seg.kvh) * kBlock);
+        row = (int)((phys * P.Hkv + seg.kvh) * P.rows_per_block);
       } else if (phys != kNotVisible) {
         if (P.dev_status) atomicOr(P.dev_status, (int)PUZZLE_DEV_BAD_BLOCK);
       }
@@ -331,24 +331,26 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
   }
 
   // ---- lane-constant shared-memory offsets
-  // FP8.  K rows for ldmatrix.x4: a lane supplies row i = lane&7 of 16-byte chunk m = lane>>3.  The 8 rows of
-  // n-tile u (u = 0, 1) of a block are tokens 4c' + 2(u ^ (c'>>1)) + e with i = 2c' + e: bank-conflict free
-  // under the 64-byte swizzle, and the accumulator columns a lane owns (2c, 2c+1 of n-tiles 0 and 1) are the
+  // FP8.  A block lands as 8 rows of 128 bytes (two tokens per row) under the 128-byte swizzle: the 16-byte
+  // chunk q of token t sits at row t/2, chunk ((t&1)*4 + q) ^ (t/2 & 7).  K rows for ldmatrix.x4: a lane
+  // supplies row i = lane&7 of chunk m = lane>>3.  The 8 rows of n-tile u (u = 0, 1) of a block are tokens
+  // 4c' + 2(u ^ (c'>>1)) + e with i = 2c' + e: bank-conflict free under that swizzle, and the accumulator columns a lane owns (2c, 2c+1 of n-tiles 0 and 1) are the
   // k-columns 2c.., 2c+8.. of its P.V A-fragment.  V rows for ldmatrix.m16n16.x2.trans.b8: lane supplies
   // matrix row (lane&15) of block (lane>>4); rows 8..15 hold tokens (row ^ 2), so that the low half of each
   // returned register is always the lane's k-columns 2c, 2c+1 and the high half its k-columns 2c+8, 2c+9.
   // bf16.  Natural order: n-tile u of a block is tokens 8u..8u+7; the 128-byte swizzle is conflict free.
-  uint32_t koff[2], vrow, vswz;
+  uint32_t koff[2], vrow, vswz, vhalf = 0;
   if constexpr (FP8) {
     const int i = lane & 7, m = lane >> 3, ci = i >> 1, e = i & 1;
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const int tok = 4 * ci + 2 * (u ^ (ci >> 1)) + e;
-      koff[u] = tok * 64 + ((m ^ ((tok >> 1) & 3)) << 4);
+      koff[u] = (tok >> 1) * 128 + (((((tok & 1) << 2) | m) ^ ((tok >> 1) & 7)) << 4);
     }
     const int vr = lane & 15, vt = vr < 8 ? vr : (vr ^ 2);
-    vrow = (lane >> 4) * BLOCK_BYTES + vt * 64;
-    vswz = (vt >> 1) & 3;
+    vrow = (lane >> 4) * BLOCK_BYTES + (vt >> 1) * 128;
+    vswz = (vt >> 1) & 7;
+    vhalf = (vt & 1) << 2;
   } else {
     // K: matrices m = lane>>3 are chunks (4h + m) of tokens 8u + (lane&7); the chunk is XOR-ed with the row
     koff[0] = (lane & 7) * 128;            // + ((chunk ^ (lane & 7)) << 4) per use
@@ -538,7 +540,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t r0, r1, r2, r3;
-            ldsm_x2_trans_b8(vbase + blk2 * 2 * BLOCK_BYTES + vrow + ((ch ^ vswz) << 4), r0, r1, r2, r3);
+            ldsm_x2_trans_b8(vbase + blk2 * 2 * BLOCK_BYTES + vrow + (((vhalf | ch) ^ vswz) << 4), r0, r1, r2, r3);
             if (edge) { r0 &= mlo; r1 &= mlo; r2 &= mhi; r3 &= mhi; }
             uint32_t b0, b1;
             e4m3x4_to_f16x2x2(r0, b0, b1);

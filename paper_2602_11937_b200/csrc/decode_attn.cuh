@@ -9,7 +9,7 @@
 namespace puzzle {
 
 struct alignas(64) DecodeParams {
-  CUtensorMap tmK;  // u8 (or bf16) [num_blocks*Hkv*16 rows][one token row], box = one 16-token block
+  CUtensorMap tmK;  // rows of 128 bytes (two FP8 tokens or one bf16 token), box = one 16-token block of one KV head
   CUtensorMap tmV;
   const __nv_bfloat16* q;
   const int32_t* block_table;
@@ -27,6 +27,7 @@ struct alignas(64) DecodeParams {
   int batch, Hkv, max_blocks_per_seq, window;
   int num_splits;  // 0 = balanced schedule
   int oob_row;     // a row coordinate outside the tensor maps: loads from it return zeros
+  int rows_per_block;  // tensor-map rows (128 bytes each) per (block, KV head): 8 (FP8) or 16 (bf16)
   float sm_scale_log2e;
 };
 
