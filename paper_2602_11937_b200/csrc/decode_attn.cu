@@ -134,18 +134,24 @@ struct Producer {
   __device__ __forceinline__ bool issue(const DecodeParams& P, const int* cum, const int* lens, int w, int lane,
                                         uint32_t stage_addr, uint32_t bar) {
     if (!ok) return false;
-    if (lane == 0) mbar_arrive_expect_tx(bar, 2 * NB * BLOCK_BYTES);
-    __syncwarp();
+    int row = P.oob_row;
     if (lane < 2 * NB) {
-      int row = P.oob_row;
       if (phys >= 0 && phys < P.num_blocks) {
         row = (int)((phys * P.Hkv + seg.kvh) * P.rows_per_block);
       } else if (phys != kNotVisible) {
         if (P.dev_status) atomicOr(P.dev_status, (int)PUZZLE_DEV_BAD_BLOCK);
       }
-      const int isv = lane / NB;
-      tma_load_2d(stage_addr + isv * (NB * BLOCK_BYTES) + (lane % NB) * BLOCK_BYTES, isv ? &P.tmV : &P.tmK, 0, row,
-                  bar);
+    }
+    // the copies are issued by one lane, which collects the row coordinates first: a TMA instruction takes
+    // warp-uniform operands, so issuing from several lanes would be serialised lane by lane anyway
+    int rows[2 * NB];
+#pragma unroll
+    for (int i = 0; i < 2 * NB; ++i) rows[i] = __shfl_sync(0xffffffffu, row, i);
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar, 2 * NB * BLOCK_BYTES);
+#pragma unroll
+      for (int i = 0; i < 2 * NB; ++i)
+        tma_load_2d(stage_addr + i * BLOCK_BYTES, i < NB ? &P.tmK : &P.tmV, 0, rows[i], bar);
     }
     if (++seg.t == seg.t_end) {
       ok = next_segment<TT>(cur, seg, P, cum, lens, w);
@@ -177,6 +183,21 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1,
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// The same with a zero C operand (first k-step of a chain): D is written, nothing has to be cleared first.
+__device__ __forceinline__ void mma_f16_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
+__device__ __forceinline__ void mma_bf16v_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                            uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 __device__ __forceinline__ void mma_bf16v(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
@@ -448,7 +469,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
       float sr[NT][2];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+        float sc[4];
         if constexpr (FP8) {
           uint32_t r[4];
           ldsm_x4(kbase + (nt >> 1) * BLOCK_BYTES + koff[nt & 1], r[0], r[1], r[2], r[3]);
@@ -456,7 +477,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
           for (int s = 0; s < 4; ++s) {
             uint32_t b0, b1;
             e4m3x4_to_f16x2x2(r[s], b0, b1);
-            mma_f16(sc, qa[s][0], 0u, qa[s][1], 0u, b0, b1);
+            if (s == 0) mma_f16_z(sc, qa[s][0], 0u, qa[s][1], 0u, b0, b1);
+            else mma_f16(sc, qa[s][0], 0u, qa[s][1], 0u, b0, b1);
           }
         } else {
 #pragma unroll
@@ -464,7 +486,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
             uint32_t r[4];
             ldsm_x4(kbase + (nt >> 1) * BLOCK_BYTES + koff[nt & 1] + (((4 * h + (lane >> 3)) ^ (lane & 7)) << 4), r[0],
                     r[1], r[2], r[3]);
-            mma_bf16v(sc, qa[2 * h][0], 0u, qa[2 * h][1], 0u, r[0], r[1]);
+            if (h == 0) mma_bf16v_z(sc, qa[2 * h][0], 0u, qa[2 * h][1], 0u, r[0], r[1]);
+            else mma_bf16v(sc, qa[2 * h][0], 0u, qa[2 * h][1], 0u, r[0], r[1]);
             mma_bf16v(sc, qa[2 * h + 1][0], 0u, qa[2 * h + 1][1], 0u, r[2], r[3]);
           }
         }
