@@ -117,25 +117,31 @@ def physical_gpu_index(local_rank: int) -> int:
 # ------------------------------------------------------------------ our arm ---
 
 def build_layer(w: synth.Workload, layer: int, dev: str):
-    """One layer's FP8 cache on the device: N(0,1) x per-head factor samples, scale = amax/448,
-    cast with the library's float8 type (input preparation, not the path under test)."""
-    nb = w.batch * w.blocks_per_seq
-    out = {}
-    for which in ("k", "v"):
-        cache = torch.empty(nb, w.hkv, w.block, w.head_dim, dtype=torch.uint8, device=dev)
-        amax = torch.zeros(w.hkv, device=dev)
-        step = 8192
-        for lo in range(0, nb, step):      # pass 1: amax per KV head
-            x = synth.draw_kv_samples(w, which, nb, layer, dev, lo, min(nb, lo + step))
-            amax = torch.maximum(amax, x.abs().amax(dim=(0, 2, 3)))
-        scale = (amax / 448.0).float()
-        scale = torch.where(scale > 0, scale, torch.ones_like(scale))
-        for lo in range(0, nb, step):      # pass 2: same draws, quantised
-            x = synth.draw_kv_samples(w, which, nb, layer, dev, lo, min(nb, lo + step))
-            cache[lo:lo + x.shape[0]] = (x / scale[None, :, None, None]).to(torch.float8_e4m3fn).view(torch.uint8)
-        out[which + "_cache"], out[which + "_scale"] = cache, scale
-    out["table"] = synth.draw_block_table(w, layer, nb, dev)
-    return out
+    """One layer's FP8 cache on the device (input preparation, see synth.device)."""
+    from synth.device import fill_layer
+    return fill_layer(w, layer, dev)
+
+
+def shard_workload(w: synth.Workload, rank: int, world: int) -> synth.Workload:
+    """Weak scaling over independent sequences: rank r of `world` runs the same shape on sequences of its
+    own (a different seed), so the job processes world x the single-GPU units with no data-path collective."""
+    if world > 1:
+        w.config_id = w.config_id + 100 * rank
+    return w
+
+
+def max_over_ranks(values, world: int, device):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the job's time)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def job_throughput_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Whole-job value: every rank moves bytes_per_rank_step per step, the step takes the slowest rank's time."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
 
 
 def run_ours(args):
@@ -150,9 +156,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    w = synth.workload(args.config)
-    if world > 1:   # weak scaling: every rank draws its own sequences
-        w.config_id = w.config_id + 100 * rank
+    w = shard_workload(synth.workload(args.config), rank, world)
     window = w.windows[0]
     seq_lens_host = synth.draw_seq_lens(w).tolist()
     seq_lens = torch.tensor(seq_lens_host, dtype=torch.int32, device=dev)
@@ -259,15 +263,12 @@ def run_ours(args):
     dev_flags = int(status.item())
     bytes_step = algorithmic_bytes(w, seq_lens_host, window)
     kv_bytes_attn = bytes_step - 2 * w.batch * w.hkv * w.head_dim * 3   # what the attention pass itself moves
-    times = torch.tensor([ms_total, ms_e2e, statistics.mean(attn_ms)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e, attn_mean_ms = (float(x) for x in times.tolist())
+    ms_total, ms_e2e, attn_mean_ms = max_over_ranks([ms_total, ms_e2e, statistics.mean(attn_ms)], world, dev)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
         ms_step = ms_total / args.steps
-        value = world * bytes_step / (ms_step * 1e-3) / 1e9
+        value = job_throughput_gbs(bytes_step, world, ms_step)
         achieved = kv_bytes_attn / (attn_mean_ms * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,

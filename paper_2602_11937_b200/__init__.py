@@ -27,3 +27,4 @@ from .binding import (  # noqa: F401
     puzzle_launch_count,
     puzzle_status_string,
 )
+from .stack import DecodeStack  # noqa: F401,E402

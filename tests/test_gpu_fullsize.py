@@ -1,0 +1,153 @@
+"""Parity at the full sizes of the benchmark workloads, in the launch configuration the bench times
+(balanced schedule, paged random block table), on sampled outputs.
+
+The caches are filled on the device (synth.device: input preparation), copied to the host bit for bit, and
+the float64 oracle recomputes a seeded sample of (sequence, query head) rows from those same bytes.  The
+append is checked on every appended byte.  Bars as in test_gpu_parity: bytes exact, |err| <= 2e-3
+(+ 2^-8 |ref| where |ref| >= 1, and everywhere on the workload whose K/V are scaled up).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from helpers import bf16_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _host(t):
+    if t is None:
+        return None
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    return t.cpu().numpy()
+
+
+class FullCase:
+    def __init__(self, w, layer, kv_dtype=oracle.KV_FP8_E4M3):
+        import paper_2602_11937_b200 as P
+        from synth.device import fill_layer
+        self.P, self.w, self.kv_dtype = P, w, kv_dtype
+        dev = "cuda"
+        self.d = fill_layer(w, layer, dev, kv_dtype)
+        self.lens_host = synth.draw_seq_lens(w).numpy().astype(np.int32)
+        self.seq_lens = torch.from_numpy(self.lens_host).to(dev)
+        self.q = synth.draw_q(w, layer, dev)
+        self.k_new, self.v_new = synth.draw_new_kv(w, layer, dev)
+        self.sinks = synth.draw_sinks(w, layer, dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.view = P.kv_view(self.d["k_cache"], self.d["v_cache"], self.seq_lens, block_table=self.d["table"],
+                              max_blocks_per_seq=w.blocks_per_seq, k_scale=self.d["k_scale"],
+                              v_scale=self.d["v_scale"])
+        self.host = None
+
+    def desc(self, window):
+        return self.P.layer_desc(window=window, kv_dtype=self.kv_dtype)
+
+    def append_and_check(self):
+        """GPU append vs oracle append on a host copy of the whole cache: every byte equal."""
+        w = self.w
+        hk, hv = _host(self.d["k_cache"]), _host(self.d["v_cache"])
+        self.P.puzzle_kv_append(self.desc(0), self.view, self.k_new, self.v_new, dev_status=self.status)
+        torch.cuda.synchronize()
+        oracle.kv_append(hk, hv, self.kv_dtype, w.block, _host(self.d["table"]), w.blocks_per_seq, self.lens_host,
+                         _host(self.d["k_scale"]), _host(self.d["v_scale"]), bf16_bits(self.k_new),
+                         bf16_bits(self.v_new))
+        gk, gv = _host(self.d["k_cache"]), _host(self.d["v_cache"])
+        assert np.array_equal(gk, hk) and np.array_equal(gv, hv), "appended bytes differ"
+        self.host = (hk, hv)
+
+    def attn_and_check(self, window, num_splits=0, n_items=16, rel=False, seed=0):
+        P, w = self.P, self.w
+        d = self.desc(window)
+        ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(d, w.batch, num_splits), dtype=torch.uint8, device="cuda")
+        P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
+        out = torch.full((w.batch, w.hq, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((w.batch, w.hq), float("nan"), dtype=torch.float32, device="cuda")
+        P.puzzle_decode_attn(d, self.view, self.q, self.sinks, out, lse, num_splits=num_splits, workspace=ws,
+                             dev_status=self.status)
+        torch.cuda.synchronize()
+        assert int(self.status.item()) == 0
+        got_all = out.float().cpu().numpy().astype(np.float64)
+        assert np.isfinite(got_all).all()
+        rng = np.random.default_rng(1000 + seed)
+        items = [(int(rng.integers(w.batch)), int(rng.integers(w.hq))) for _ in range(n_items)]
+        items += [(int(np.argmax(self.lens_host)), 0), (int(np.argmin(self.lens_host)), w.hq - 1)]
+        hk, hv = self.host
+        ref, ref_lse = oracle.decode_attn(hk, hv, self.kv_dtype, _host(self.d["table"]), w.blocks_per_seq,
+                                          self.lens_host, _host(self.d["k_scale"]), _host(self.d["v_scale"]),
+                                          bf16_bits(self.q), _host(self.sinks), window, w.head_dim ** -0.5, items=items)
+        got = np.stack([got_all[b, h] for b, h in items])
+        got_lse = np.array([lse[b, h].item() for b, h in items])
+        a = np.abs(ref)
+        bound = 2e-3 + np.where((a >= 1.0) | rel, 2.0 ** -8 * a, 0.0)
+        err = np.abs(got - ref)
+        assert (err <= bound).all(), "max |err| %.3e over bound at W=%d S=%d" % (err.max(), window, num_splits)
+        assert np.all(np.abs(got_lse - ref_lse) <= 2e-3)
+        return float(err.max())
+
+
+def test_full_size_64k_context_split_sweep():
+    """Batch 16, context 65536, full attention, K/V scaled per head by U[0.5, 4]; balanced schedule and the
+    ends of the explicit split sweep."""
+    case = FullCase(synth.workload(3), 0)
+    case.append_and_check()
+    for s in (0, 8, 128):
+        case.attn_and_check(0, num_splits=s, rel=True, seed=s)
+
+
+def test_full_size_ragged_stack_layers():
+    """Batch 64, ragged contexts in [16K, 48K]: one cache, the three layer kinds of the 36-layer patterns."""
+    case = FullCase(synth.workload(4), 1)
+    case.append_and_check()
+    for window in (0, 128, 8192):
+        case.attn_and_check(window, seed=window)
+
+
+@pytest.mark.parametrize("kv_dtype", [oracle.KV_FP8_E4M3, oracle.KV_BF16], ids=["fp8", "bf16"])
+def test_full_size_128k_context(kv_dtype):
+    """Batch 8, context 131072: FP8 cache, and the bf16 cache of the same samples."""
+    case = FullCase(synth.workload(5), 1, kv_dtype)
+    case.append_and_check()
+    case.attn_and_check(0, seed=1)
+    case.attn_and_check(128, seed=2)
+
+
+def test_stack_driver_matches_layer_by_layer_calls():
+    """The per-layer pattern driver (eager and as a CUDA graph) gives what the single calls give."""
+    import paper_2602_11937_b200 as P
+    from synth.device import fill_layer
+    w = synth.workload(4, scale=0.03)                     # batch 2, ragged contexts up to 1475
+    windows = [128, 0, 8192, 0]
+    L = [fill_layer(w, i, "cuda") for i in range(len(windows))]
+    seq = synth.draw_seq_lens(w, "cuda")
+    q = [synth.draw_q(w, i, "cuda") for i in range(len(windows))]
+    kv = [synth.draw_new_kv(w, i, "cuda") for i in range(len(windows))]
+    sinks = [synth.draw_sinks(w, i, "cuda") for i in range(len(windows))]
+    stack = P.DecodeStack(windows, [x["k_cache"] for x in L], [x["v_cache"] for x in L], seq,
+                          [x["table"] for x in L], w.blocks_per_seq, [x["k_scale"] for x in L],
+                          [x["v_scale"] for x in L], sinks)
+    ref = []
+    for i, win in enumerate(windows):
+        d = P.layer_desc(window=win)
+        ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(d, w.batch, 0), dtype=torch.uint8, device="cuda")
+        o = torch.empty(w.batch, w.hq, w.head_dim, dtype=torch.bfloat16, device="cuda")
+        P.puzzle_kv_append(d, stack.views[i], kv[i][0], kv[i][1])
+        P.puzzle_decode_attn(d, stack.views[i], q[i], sinks[i], o, None, workspace=ws)
+        ref.append(o)
+    out = [torch.zeros_like(r) for r in ref]
+    stack.step(q, [a for a, _ in kv], [b for _, b in kv], out)
+    torch.cuda.synchronize()
+    for o, r in zip(out, ref):
+        assert torch.equal(o, r)
+    out2 = [torch.zeros_like(r) for r in ref]
+    g = stack.capture(q, [a for a, _ in kv], [b for _, b in kv], out2)
+    for o in out2:
+        o.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    for o, r in zip(out2, ref):
+        assert torch.equal(o, r)
+    assert int(stack.status.item()) == 0
