@@ -327,6 +327,63 @@ def cpu_baseline(w, layer, seq_lens_host, q, sinks, window, pairs: int = 128):
                 pairs, w.batch * w.hkv, w.context)}
 
 
+# ------------------------------------------------------- 36-layer stack mode ---
+
+def run_stack(args):
+    """One decode step of the 36-layer attention stack (workload 4 or 5) under a per-layer pattern, as one
+    CUDA graph: append + attention per layer.  Prints its own JSON line (not the headline metric)."""
+    import paper_2602_11937_b200 as P
+    from synth.device import fill_layer, KV_BF16, KV_FP8_E4M3
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    kv_dtype = KV_BF16 if args.kv == "bf16" else KV_FP8_E4M3
+    w = synth.workload(args.stack, pattern=args.pattern)
+    windows = w.windows
+    seq_lens_host = synth.draw_seq_lens(w).tolist()
+    seq_lens = torch.tensor(seq_lens_host, dtype=torch.int32, device=dev)
+    # every full-context layer gets a cache of its own; the window layers of one size share one pool cache but
+    # each has its own random block table into it, so no two layers touch the same bytes
+    pools, layers = {}, []
+    for i, win in enumerate(windows):
+        if win == 0:
+            layers.append(fill_layer(w, i, dev, kv_dtype))
+        else:
+            if win not in pools:
+                pools[win] = fill_layer(w, 1000 + win, dev, kv_dtype, with_table=False)
+            L = dict(pools[win])
+            L["table"] = synth.draw_block_table(w, i, w.batch * w.blocks_per_seq, dev)
+            layers.append(L)
+    q = [synth.draw_q(w, i, dev) for i in range(len(windows))]
+    kv = [synth.draw_new_kv(w, i, dev) for i in range(len(windows))]
+    sinks = [synth.draw_sinks(w, i, dev) for i in range(len(windows))]
+    out = [torch.empty(w.batch, w.hq, w.head_dim, dtype=torch.bfloat16, device=dev) for _ in windows]
+    stack = P.DecodeStack(windows, [L["k_cache"] for L in layers], [L["v_cache"] for L in layers], seq_lens,
+                          [L["table"] for L in layers], w.blocks_per_seq, [L["k_scale"] for L in layers],
+                          [L["v_scale"] for L in layers], sinks, kv_dtype=kv_dtype)
+    g = stack.capture(q, [a for a, _ in kv], [b for _, b in kv], out)
+    for _ in range(max(args.warmup, 3)):
+        g.replay()
+    torch.cuda.synchronize()
+    steps = min(args.steps, 200)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        g.replay()
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / steps
+    nbytes = sum(algorithmic_bytes(w, seq_lens_host, win, fp8=kv_dtype == KV_FP8_E4M3) for win in windows)
+    peak, kind = measured_peak()
+    print(json.dumps({
+        "metric": "decode_attn_stack_step", "workload": w.name, "kv": args.kv, "layers": len(windows),
+        "full_layers": sum(1 for x in windows if x == 0), "window_sizes": sorted(set(x for x in windows if x)),
+        "us_per_step": round(ms * 1e3, 1), "us_per_layer": round(ms * 1e3 / len(windows), 2),
+        "algorithmic_gib_per_step": round(nbytes / 2 ** 30, 3), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+        "frac_of_" + kind: round(nbytes / (ms * 1e-3) / 1e9 / peak, 4), "steps": steps, "cuda_graph": True,
+        "dev_status": int(stack.status.item())}))
+
+
 # ------------------------------------------------------------ reference arm ---
 
 def run_reference(args):
@@ -387,13 +444,19 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="workload id 1..5 (3 = batch 16, context 64K)")
     ap.add_argument("--splits", type=int, default=0, help="0 = balanced schedule, S = fixed splits per sequence")
     ap.add_argument("--layers", type=int, default=4, help="distinct layer caches rotated between steps")
+    ap.add_argument("--stack", type=int, default=0, choices=[0, 4, 5],
+                    help="instead of the headline run: one step of the 36-layer stack of workload 4 or 5")
+    ap.add_argument("--pattern", default="parent", choices=["parent", "every4th", "selective"])
+    ap.add_argument("--kv", default="fp8", choices=["fp8", "bf16"])
     ap.add_argument("--contiguous", action="store_true",
                     help="diagnostic: drop the block table (sequence b owns blocks b*blocks_per_seq ...)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--ncu-traffic", type=float, default=None,
                     help="DRAM bytes per launch of the attention kernel from an ncu capture (reported as-is)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.stack:
+        run_stack(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
