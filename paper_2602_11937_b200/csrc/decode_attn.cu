@@ -32,6 +32,8 @@
 //    and writes the bf16 output: one launch per layer, no waiting anywhere.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "decode_attn.cuh"
 
@@ -381,6 +383,22 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     vswz = lane & 7;                        // row & 7
   }
 
+  // per-use lane-constant offsets, hoisted: inside the tile loop an address is stage base + one of these,
+  // the block offset goes into the instruction as an immediate
+  uint32_t kof[2][2], vof[4];
+  if constexpr (FP8) {
+    kof[0][0] = koff[0]; kof[1][0] = koff[1]; kof[0][1] = 0; kof[1][1] = 0;
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) vof[ch] = vrow + (((vhalf | ch) ^ vswz) << 4);
+  } else {
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) kof[u][h] = koff[u] + (((4 * h + (lane >> 3)) ^ (lane & 7)) << 4);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) vof[j] = vrow + (((2 * j + (lane >> 4)) ^ vswz) << 4);
+  }
+
   Producer<TT> prod;
   prod.start(cc, P, cum, lens, w, lane);
   int inflight = 0;
@@ -464,6 +482,11 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
       const uint32_t vbase = kbase + NB * BLOCK_BYTES;
       const int tok0 = t * TT;
       const bool edge = (tok0 < cs.lo) || (tok0 + TT > cs.L);
+      const uint32_t kb[2][2] = {{kbase + kof[0][0], kbase + kof[0][1]}, {kbase + kof[1][0], kbase + kof[1][1]}};
+      const uint32_t vb[4] = {vbase + vof[0], vbase + vof[1], vbase + vof[2], vbase + vof[3]};
+      // the tile's math, compiled twice: interior tiles carry none of the masking of edge tiles
+      auto tile_math = [&](auto edge_tag) {
+      constexpr bool EDGE = decltype(edge_tag)::value;
 
       // ---- S^T[head][token] = Q K^T (code products; the scales are folded into alpha)
       float sr[NT][2];
@@ -472,7 +495,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
         float sc[4];
         if constexpr (FP8) {
           uint32_t r[4];
-          ldsm_x4(kbase + (nt >> 1) * BLOCK_BYTES + koff[nt & 1], r[0], r[1], r[2], r[3]);
+          ldsm_x4(kb[nt & 1][0] + (nt >> 1) * BLOCK_BYTES, r[0], r[1], r[2], r[3]);
 #pragma unroll
           for (int s = 0; s < 4; ++s) {
             uint32_t b0, b1;
@@ -484,8 +507,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
 #pragma unroll
           for (int h = 0; h < 2; ++h) {  // dims 32h .. 32h+31: chunks 4h .. 4h+3
             uint32_t r[4];
-            ldsm_x4(kbase + (nt >> 1) * BLOCK_BYTES + koff[nt & 1] + (((4 * h + (lane >> 3)) ^ (lane & 7)) << 4), r[0],
-                    r[1], r[2], r[3]);
+            ldsm_x4(kb[nt & 1][h] + (nt >> 1) * BLOCK_BYTES, r[0], r[1], r[2], r[3]);
             if (h == 0) mma_bf16v_z(sc, qa[2 * h][0], 0u, qa[2 * h][1], 0u, r[0], r[1]);
             else mma_bf16v(sc, qa[2 * h][0], 0u, qa[2 * h][1], 0u, r[0], r[1]);
             mma_bf16v(sc, qa[2 * h + 1][0], 0u, qa[2 * h + 1][1], 0u, r[2], r[3]);
@@ -494,7 +516,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
         sr[nt][0] = sc[0];
         sr[nt][1] = sc[1];
       }
-      if (edge) {
+      if constexpr (EDGE) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const int tk = tok0 + (nt >> 1) * kBlock + (FP8 ? 4 * c + 2 * ((nt & 1) ^ (c >> 1)) : 8 * (nt & 1) + 2 * c);
@@ -550,7 +572,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
       for (int blk2 = 0; blk2 < NB / 2; ++blk2) {
         if constexpr (FP8) {
           uint32_t mlo = 0xffffffffu, mhi = 0xffffffffu;
-          if (edge) {  // zero the V codes of tokens at or beyond L (they may hold anything, NaN codes included)
+          if constexpr (EDGE) {  // zero the V codes of tokens at or beyond L (they may hold anything, NaN codes included)
             const int n0 = cs.L - (tok0 + 32 * blk2 + 4 * c);
             const int n1 = n0 - kBlock;
             mlo = n0 >= 4 ? 0xffffffffu : (n0 <= 0 ? 0u : (1u << (8 * n0)) - 1u);
@@ -563,8 +585,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t r0, r1, r2, r3;
-            ldsm_x2_trans_b8(vbase + blk2 * 2 * BLOCK_BYTES + vrow + (((vhalf | ch) ^ vswz) << 4), r0, r1, r2, r3);
-            if (edge) { r0 &= mlo; r1 &= mlo; r2 &= mhi; r3 &= mhi; }
+            ldsm_x2_trans_b8(vb[ch] + blk2 * 2 * BLOCK_BYTES, r0, r1, r2, r3);
+            if constexpr (EDGE) { r0 &= mlo; r1 &= mlo; r2 &= mhi; r3 &= mhi; }
             uint32_t b0, b1;
             e4m3x4_to_f16x2x2(r0, b0, b1);
             mma_f16(O[2 * ch], pa[2 * blk2][0], pa[2 * blk2][1], pa[2 * blk2][2], pa[2 * blk2][3], b0, b1);
@@ -582,7 +604,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
           for (int bb = 0; bb < 2; ++bb) {
             const int blk = 2 * blk2 + bb;
             uint32_t mlo = 0xffffffffu, mhi = 0xffffffffu;
-            if (edge) {  // zero the V values of tokens at or beyond L
+            if constexpr (EDGE) {  // zero the V values of tokens at or beyond L
               const int n0 = cs.L - (tok0 + kBlock * blk + 2 * c);
               const int n1 = n0 - 8;
               mlo = n0 >= 2 ? 0xffffffffu : (n0 <= 0 ? 0u : 0xffffu);
@@ -591,14 +613,17 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
 #pragma unroll
             for (int j = 0; j < 4; ++j) {  // dim chunks 2j, 2j+1 -> n-tiles 2j, 2j+1
               uint32_t r0, r1, r2, r3;
-              ldsm_x4_trans(vbase + blk * BLOCK_BYTES + vrow + (((2 * j + (lane >> 4)) ^ vswz) << 4), r0, r1, r2, r3);
-              if (edge) { r0 &= mlo; r1 &= mhi; r2 &= mlo; r3 &= mhi; }
+              ldsm_x4_trans(vb[j] + blk * BLOCK_BYTES, r0, r1, r2, r3);
+              if constexpr (EDGE) { r0 &= mlo; r1 &= mhi; r2 &= mlo; r3 &= mhi; }
               mma_bf16v(O[2 * j], pa[blk][0], pa[blk][1], pa[blk][2], pa[blk][3], r0, r1);
               mma_bf16v(O[2 * j + 1], pa[blk][0], pa[blk][1], pa[blk][2], pa[blk][3], r2, r3);
             }
           }
         }
       }
+
+      };  // tile_math
+      if (edge) tile_math(std::true_type{}); else tile_math(std::false_type{});
 
       // ---- refill this stage with the tile NS ahead
       __syncwarp();
