@@ -173,6 +173,13 @@ def run_ours(args):
     k_new, v_new = synth.draw_new_kv(w, 0, dev)
     sinks = synth.draw_sinks(w, 0, dev)
     out = torch.empty(w.batch, w.hq, w.head_dim, dtype=torch.bfloat16, device=dev)
+    decode = P.puzzle_decode_attn_tcgen05 if args.kernel == "tcgen05" else P.puzzle_decode_attn
+    if args.kernel == "tcgen05":
+        kernel_name = "decode_attn_tc_kernel (tcgen05 split-KV pass with the merge fused in)"
+        dtype_name = "e4m3 tcgen05 mma on the cache codes, f32 accumulate and softmax"
+    else:
+        kernel_name = "decode_attn_kernel<fp8> (split-KV pass with the merge fused in)"
+        dtype_name = "f16 mma on e4m3 codes, f32 accumulate and softmax"
     ws = torch.empty(P.puzzle_decode_attn_workspace_bytes(desc, w.batch, args.splits), dtype=torch.uint8, device=dev)
     P.puzzle_decode_attn_workspace_init(desc, w.batch, ws)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -181,7 +188,7 @@ def run_ours(args):
     def step(i):
         v = views[i % len(views)]
         P.puzzle_kv_append(desc, v, k_new, v_new, dev_status=status, stream=stream)
-        P.puzzle_decode_attn(desc, v, q, sinks, out, None, num_splits=args.splits, workspace=ws,
+        decode(desc, v, q, sinks, out, None, num_splits=args.splits, workspace=ws,
                              dev_status=status, stream=stream)
 
     def barrier():
@@ -212,7 +219,7 @@ def run_ours(args):
     a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a0.record(stream)
     for i in range(n_attn):
-        P.puzzle_decode_attn(desc, views[i % len(views)], q, sinks, out, None, num_splits=args.splits, workspace=ws,
+        decode(desc, views[i % len(views)], q, sinks, out, None, num_splits=args.splits, workspace=ws,
                              dev_status=status, stream=stream)
     a1.record(stream)
     barrier()
@@ -228,7 +235,7 @@ def run_ours(args):
         v = views[i % len(views)]
         dq.copy_(hq_, non_blocking=True); dk.copy_(hk_, non_blocking=True); dv.copy_(hv_, non_blocking=True)
         P.puzzle_kv_append(desc, v, dk, dv, dev_status=status, stream=stream)
-        P.puzzle_decode_attn(desc, v, dq, sinks, out, None, num_splits=args.splits, workspace=ws,
+        decode(desc, v, dq, sinks, out, None, num_splits=args.splits, workspace=ws,
                              dev_status=status, stream=stream)
         hout.copy_(out, non_blocking=True)
 
@@ -274,7 +281,7 @@ def run_ours(args):
             "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5),
             "us_per_layer_step": round(ms_step * 1e3, 2), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f16 mma on e4m3 codes, f32 accumulate and softmax", "data": "synthetic",
+            "vs_baseline": None, "dtype": dtype_name, "data": "synthetic",
             "config": {"workload": w.name, "batch_per_gpu": w.batch, "context": w.context, "q_heads": w.hq,
                        "kv_heads": w.hkv, "head_dim": w.head_dim, "block_size": w.block, "window": window, "paged": not args.contiguous,
                        "num_splits": args.splits, "rotating_layer_caches": len(layers),
@@ -287,7 +294,7 @@ def run_ours(args):
                     "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in (q, k_new, v_new))),
                     "d2h_bytes_per_step": int(out.numel() * out.element_size())},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "decode_attn_kernel<fp8> (split-KV pass with the merge fused in)",
+            "roofline": {"bound": "hbm", "kernel": kernel_name,
                          "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
                          "unit": "GB/s", "frac": round(achieved / peak, 4),
                          "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
@@ -448,6 +455,8 @@ def main():
                     help="instead of the headline run: one step of the 36-layer stack of workload 4 or 5")
     ap.add_argument("--pattern", default="parent", choices=["parent", "every4th", "selective"])
     ap.add_argument("--kv", default="fp8", choices=["fp8", "bf16"])
+    ap.add_argument("--kernel", default="mma", choices=["mma", "tcgen05"],
+                    help="split-KV kernel of the headline run: mma.sync (default) or the tcgen05 / tensor-memory one")
     ap.add_argument("--contiguous", action="store_true",
                     help="diagnostic: drop the block table (sequence b owns blocks b*blocks_per_seq ...)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")

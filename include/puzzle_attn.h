@@ -139,6 +139,21 @@ PUZZLE_API puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const
                                  int32_t num_splits, void* workspace, size_t workspace_bytes,
                                  int32_t* dev_status, void* stream);
 
+/* The same operation and contract as puzzle_decode_attn (same arguments, same workspace, same
+ * results within the same tolerance), computed by a second kernel that feeds the E4M3 codes of the
+ * cache straight to the 5th-generation tensor cores (tcgen05 MMA, accumulators in tensor memory):
+ * S = K Q^T with the bf16 query split exactly into two E4M3 terms, O^T += V^T P with the softmax
+ * weights split into four E4M3 terms.  FP8 caches only: a bf16 cache returns
+ * PUZZLE_ERR_UNSUPPORTED and nothing is launched.  Tiles are 128 tokens (num_splits >= 1 cuts the
+ * context into runs of 128-token tiles).  It is the slower of the two kernels on the workloads
+ * measured so far and is kept as a validated alternative; puzzle_decode_attn is the default path.
+ * (Paper: KV-cache I/O bounds decoding, Section "Optimized Scenarios"; FP8 KV cache, Section
+ * "KV Quantization".) */
+PUZZLE_API puzzle_status puzzle_decode_attn_tcgen05(const puzzle_layer_desc* desc, const puzzle_kv_view* kv,
+                                 const void* q, const float* sinks, void* out, float* lse_out, int32_t batch,
+                                 int32_t num_splits, void* workspace, size_t workspace_bytes,
+                                 int32_t* dev_status, void* stream);
+
 /* Size of the scratch array built into the library for puzzle_decode_attn_static. */
 #define PUZZLE_STATIC_SCRATCH_BYTES (8u << 20)
 

@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     puzzle_attn_merge,
     puzzle_decode_attn,
     puzzle_decode_attn_static,
+    puzzle_decode_attn_tcgen05,
     puzzle_decode_attn_workspace_bytes,
     puzzle_decode_attn_workspace_init,
     puzzle_hbm_read_probe,

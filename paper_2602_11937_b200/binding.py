@@ -24,6 +24,7 @@ EXPORTS = (
     "puzzle_decode_attn_workspace_bytes",
     "puzzle_decode_attn_workspace_init",
     "puzzle_decode_attn",
+    "puzzle_decode_attn_tcgen05",
     "puzzle_decode_attn_static",
     "puzzle_attn_merge",
     "puzzle_hbm_read_probe",
@@ -72,6 +73,8 @@ def _load():
         lib.puzzle_decode_attn.restype = ctypes.c_int
         lib.puzzle_decode_attn.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp, i32, i32,
                                            vp, sz, vp, vp]
+        lib.puzzle_decode_attn_tcgen05.restype = ctypes.c_int
+        lib.puzzle_decode_attn_tcgen05.argtypes = lib.puzzle_decode_attn.argtypes
         lib.puzzle_decode_attn_static.restype = ctypes.c_int
         lib.puzzle_decode_attn_static.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp,
                                                   i32, i32, vp, vp]
@@ -165,18 +168,32 @@ def puzzle_decode_attn_workspace_init(desc: LayerDesc, batch: int, workspace: to
            "puzzle_decode_attn_workspace_init")
 
 
+def _decode_attn(name: str, desc: LayerDesc, view: KVView, q, sinks, out, lse_out, num_splits, workspace, dev_status,
+                 stream) -> None:
+    batch = q.shape[0]
+    if workspace is None:
+        raise ValueError("workspace is required (size it with puzzle_decode_attn_workspace_bytes)")
+    _check(getattr(_load(), name)(ctypes.byref(desc), ctypes.byref(view), _p(q, torch.bfloat16, "q"),
+                                  _p(sinks, torch.float32, "sinks"), _p(out, torch.bfloat16, "out"),
+                                  _p(lse_out, torch.float32, "lse_out"), batch, int(num_splits), _p(workspace),
+                                  workspace.numel() * workspace.element_size(), _p(dev_status, torch.int32),
+                                  _stream(stream)), name)
+
+
 def puzzle_decode_attn(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Optional[torch.Tensor],
                        out: torch.Tensor, lse_out: Optional[torch.Tensor] = None, num_splits: int = 0,
                        workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
                        stream=None) -> None:
-    batch = q.shape[0]
-    if workspace is None:
-        raise ValueError("workspace is required (size it with puzzle_decode_attn_workspace_bytes)")
-    _check(_load().puzzle_decode_attn(ctypes.byref(desc), ctypes.byref(view), _p(q, torch.bfloat16, "q"),
-                                      _p(sinks, torch.float32, "sinks"), _p(out, torch.bfloat16, "out"),
-                                      _p(lse_out, torch.float32, "lse_out"), batch, int(num_splits), _p(workspace),
-                                      workspace.numel() * workspace.element_size(), _p(dev_status, torch.int32),
-                                      _stream(stream)), "puzzle_decode_attn")
+    _decode_attn("puzzle_decode_attn", desc, view, q, sinks, out, lse_out, num_splits, workspace, dev_status, stream)
+
+
+def puzzle_decode_attn_tcgen05(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Optional[torch.Tensor],
+                               out: torch.Tensor, lse_out: Optional[torch.Tensor] = None, num_splits: int = 0,
+                               workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                               stream=None) -> None:
+    """puzzle_decode_attn computed by the tcgen05 / tensor-memory kernel (FP8 caches only)."""
+    _decode_attn("puzzle_decode_attn_tcgen05", desc, view, q, sinks, out, lse_out, num_splits, workspace, dev_status,
+                 stream)
 
 
 def puzzle_decode_attn_static(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Optional[torch.Tensor],

@@ -31,7 +31,7 @@ EncodeTiledFn encode_tiled() {
 
 struct DeviceInfo {
   int sm_count = 0;
-  int smem_limit[2] = {0, 0};  // per split-KV kernel variant (FP8, bf16); 0 = not raised yet
+  int smem_limit[3] = {0, 0, 0};  // per split-KV kernel (FP8 mma.sync, bf16, FP8 tensor-memory); 0 = not raised yet
 };
 DeviceInfo& device_info() {
   static DeviceInfo info[64];
@@ -67,9 +67,19 @@ puzzle_status check_view(const puzzle_layer_desc* d, const puzzle_kv_view* kv, i
 
 // 2-D view of a cache as rows of 128 bytes: two FP8 tokens or one bf16 token per row, so that every TMA
 // request is a full 128-byte line.  Box = one 16-token block of one KV head (8 or 16 rows), 128-byte swizzle.
-bool make_cache_map(CUtensorMap* m, void* base, long long rows, int elem_bytes) {
+// row_bytes = 64 (FP8 only): one token per row, 16 rows per block, 64-byte swizzle (the tensor-memory kernel's view).
+bool make_cache_map(CUtensorMap* m, void* base, long long rows, int elem_bytes, int row_bytes = 128) {
   EncodeTiledFn enc = encode_tiled();
   if (!enc) return false;
+  if (row_bytes == 64) {
+    const cuuint64_t dims[2] = {64, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {64};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kBlock};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  }
   const cuuint64_t inner = 128 / elem_bytes;  // elements per row
   const cuuint64_t dims[2] = {inner, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {128};
@@ -139,9 +149,10 @@ size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t
          workspace_floats(batch, desc->num_kv_heads, num_splits, desc->kv_dtype) * sizeof(float);
 }
 
-puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
-                                 const float* sinks, void* out, float* lse_out, int32_t batch, int32_t num_splits,
-                                 void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                      const float* sinks, void* out, float* lse_out, int32_t batch,
+                                      int32_t num_splits, void* workspace, size_t workspace_bytes,
+                                      int32_t* dev_status, void* stream, bool tcgen05) {
   puzzle_status st = check_desc(desc);
   if (st != PUZZLE_OK) return st;
   st = check_view(desc, kv, batch);
@@ -165,9 +176,13 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   DecodeParams P;
   std::memset(&P, 0, sizeof P);
   const int eb = fp8 ? 1 : 2;
-  const int rows_per_block = kBlock * kHeadDim * eb / 128;
+  if (tcgen05 && !fp8) return PUZZLE_ERR_UNSUPPORTED;   // the tensor-memory kernel reads E4M3 codes only
+  const bool tc = tcgen05;
+  const int row_bytes = tc ? 64 : 128;
+  const int rows_per_block = kBlock * kHeadDim * eb / row_bytes;
   const long long cache_rows = kv->num_blocks * Hkv * (long long)rows_per_block;
-  if (!make_cache_map(&P.tmK, kv->k_cache, cache_rows, eb) || !make_cache_map(&P.tmV, kv->v_cache, cache_rows, eb))
+  if (!make_cache_map(&P.tmK, kv->k_cache, cache_rows, eb, row_bytes) ||
+      !make_cache_map(&P.tmV, kv->v_cache, cache_rows, eb, row_bytes))
     return PUZZLE_ERR_CUDA;
   P.q = static_cast<const __nv_bfloat16*>(q);
   P.block_table = kv->block_table;
@@ -191,10 +206,27 @@ puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_
   P.rows_per_block = rows_per_block;
   P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
 
-  if (launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit) != cudaSuccess) return PUZZLE_ERR_CUDA;
+  const cudaError_t le = tc ? launch_decode_attn_tc(P, ctas, s, device_info().smem_limit + 2)
+                            : launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
+  if (le != cudaSuccess) return PUZZLE_ERR_CUDA;
   count_launch();
 
   return PUZZLE_OK;
+}
+
+puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                 const float* sinks, void* out, float* lse_out, int32_t batch, int32_t num_splits,
+                                 void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+  return decode_attn_impl(desc, kv, q, sinks, out, lse_out, batch, num_splits, workspace, workspace_bytes, dev_status,
+                          stream, false);
+}
+
+puzzle_status puzzle_decode_attn_tcgen05(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                         const float* sinks, void* out, float* lse_out, int32_t batch,
+                                         int32_t num_splits, void* workspace, size_t workspace_bytes,
+                                         int32_t* dev_status, void* stream) {
+  return decode_attn_impl(desc, kv, q, sinks, out, lse_out, batch, num_splits, workspace, workspace_bytes, dev_status,
+                          stream, true);
 }
 
 puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_desc* desc, int32_t batch, void* workspace,

@@ -54,6 +54,10 @@ constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
 // Launches the split-KV kernel for an FP8 (fp8 = true) or bf16 cache on `ctas` CTAs.  smem_limit[2] caches,
 // per variant, the dynamic shared-memory limit set for the kernel on the current device (0 = not set yet).
 cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit);
+// The tensor-memory (tcgen05) kernel for the FP8 cache.  Its tensor maps view the cache as rows of 64 bytes
+// (one token), box = 16 rows, 64-byte swizzle; P.rows_per_block is 16 and P.oob_row counts such rows.
+cudaError_t launch_decode_attn_tc(const DecodeParams& P, int ctas, cudaStream_t s, int* smem_limit);
+int decode_attn_tc_workers_per_cta();
 
 __global__ void attn_merge_kernel(const MergeParams P);
 

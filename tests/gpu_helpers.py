@@ -53,7 +53,7 @@ class DeviceCase:
         P.puzzle_kv_append(self.desc(), self.view(), self.k_new, self.v_new, dev_status=self.status)
         torch.cuda.synchronize()
 
-    def attn(self, window=0, num_splits=0, sinks="case", seq_lens=None, want_lse=True):
+    def attn(self, window=0, num_splits=0, sinks="case", seq_lens=None, want_lse=True, kernel="mma"):
         w = self.w
         d = self.desc(window)
         ws = torch.empty(max(16, P.puzzle_decode_attn_workspace_bytes(d, w.batch, num_splits)), dtype=torch.uint8,
@@ -63,8 +63,8 @@ class DeviceCase:
         out = torch.full((w.batch, w.hq, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
         lse = torch.full((w.batch, w.hq), float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
         s = self.sinks if isinstance(sinks, str) else sinks
-        P.puzzle_decode_attn(d, self.view(seq_lens), self.q, s, out, lse, num_splits=num_splits, workspace=ws,
-                             dev_status=self.status)
+        call = P.puzzle_decode_attn_tcgen05 if kernel == "tcgen05" else P.puzzle_decode_attn
+        call(d, self.view(seq_lens), self.q, s, out, lse, num_splits=num_splits, workspace=ws, dev_status=self.status)
         torch.cuda.synchronize()
         return out.float().cpu().numpy().astype(np.float64), (None if lse is None else lse.cpu().numpy().astype(np.float64))
 

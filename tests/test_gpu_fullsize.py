@@ -59,15 +59,15 @@ class FullCase:
         assert np.array_equal(gk, hk) and np.array_equal(gv, hv), "appended bytes differ"
         self.host = (hk, hv)
 
-    def attn_and_check(self, window, num_splits=0, n_items=16, rel=False, seed=0):
+    def attn_and_check(self, window, num_splits=0, n_items=16, rel=False, seed=0, kernel="mma"):
         P, w = self.P, self.w
         d = self.desc(window)
         ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(d, w.batch, num_splits), dtype=torch.uint8, device="cuda")
         P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
         out = torch.full((w.batch, w.hq, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
         lse = torch.full((w.batch, w.hq), float("nan"), dtype=torch.float32, device="cuda")
-        P.puzzle_decode_attn(d, self.view, self.q, self.sinks, out, lse, num_splits=num_splits, workspace=ws,
-                             dev_status=self.status)
+        call = P.puzzle_decode_attn_tcgen05 if kernel == "tcgen05" else P.puzzle_decode_attn
+        call(d, self.view, self.q, self.sinks, out, lse, num_splits=num_splits, workspace=ws, dev_status=self.status)
         torch.cuda.synchronize()
         assert int(self.status.item()) == 0
         got_all = out.float().cpu().numpy().astype(np.float64)

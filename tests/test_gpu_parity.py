@@ -84,14 +84,14 @@ def test_append_bf16_cache_is_a_copy():
 
 # --------------------------------------------------------------- attention ---
 
-def _run_and_compare(case, window, num_splits=0, rel=False, sinks="case"):
+def _run_and_compare(case, window, num_splits=0, rel=False, sinks="case", kernel="mma"):
     from gpu_helpers import assert_close
     dev = _dev(case)
     dev.append()
     oracle_append(case)
     gk, gv = dev.cache_bytes()
     assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
-    got, got_lse = dev.attn(window=window, num_splits=num_splits, sinks=sinks)
+    got, got_lse = dev.attn(window=window, num_splits=num_splits, sinks=sinks, kernel=kernel)
     s = case["sinks"] if isinstance(sinks, str) else (None if sinks is None else sinks.cpu().numpy())
     ref, ref_lse = oracle_attn(case, window, sinks=s)
     assert int(dev.status.item()) == 0
