@@ -90,6 +90,25 @@ typedef struct {
   const float* v_scale;
 } puzzle_kv_view;
 
+/* Max calibration of the per-head scales, step 1 (paper Section "KV Quantization": FP8 KV cache with
+ * scales from max calibration).  Raises amax[h] to the largest |x| over every token and channel of KV
+ * head h of this tensor: amax[h] = max(amax[h], max_{t,d} |x[t][h][d]|).  NaNs are skipped, infinities
+ * count.  Call it once per chunk of calibration data; start from amax = 0.
+ *   x: device, bf16 [n_tokens][num_kv_heads][head_dim], 16-byte aligned; head_dim a multiple of 8;
+ *   amax: device, float32 [num_kv_heads], read and written (values must be >= 0);
+ *   num_kv_heads <= 64.  n_tokens == 0 is legal and launches nothing.
+ * Errors: PUZZLE_ERR_NULL, PUZZLE_ERR_SHAPE (sizes, alignment) before any launch. */
+PUZZLE_API puzzle_status puzzle_kv_amax_update(const void* x, int64_t n_tokens, int32_t num_kv_heads,
+                                 int32_t head_dim, float* amax, void* stream);
+
+/* Max calibration, step 2: scale[h] = amax[h] / 448 as an IEEE float32 quotient (448 = largest E4M3
+ * value), so that x / scale fills the E4M3 range; amax[h] == 0 gives scale 1.  pow2 != 0 rounds every
+ * scale up to the next power of two (a power of two stays), as the paper does ("rounded the scales up
+ * to a power of 2", same Section).  These are the dequantisation scales puzzle_kv_view carries
+ * (x ~ code * scale).  amax and scale_out: device float32 [num_kv_heads]; they may be the same array. */
+PUZZLE_API puzzle_status puzzle_kv_scales_from_amax(const float* amax, int32_t num_kv_heads, int32_t pow2,
+                                 float* scale_out, void* stream);
+
 /* Quantise-and-append of the new token's K and V (one token per sequence).
  * FP8: code = E4M3(round-to-nearest-even, saturating at +-448, of the float32
  * quotient x / scale[h]); NaN -> 0x7F.  bf16: the value is copied.  The token

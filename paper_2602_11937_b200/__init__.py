@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     KVView,
     LayerDesc,
     PuzzleError,
+    calibrate_scales,
     kv_view,
     layer_desc,
     library_path,
@@ -24,7 +25,9 @@ from .binding import (  # noqa: F401
     puzzle_decode_attn_workspace_bytes,
     puzzle_decode_attn_workspace_init,
     puzzle_hbm_read_probe,
+    puzzle_kv_amax_update,
     puzzle_kv_append,
+    puzzle_kv_scales_from_amax,
     puzzle_launch_count,
     puzzle_status_string,
 )

@@ -20,6 +20,8 @@ DEV_WAIT_EXPIRED = 4
 STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = (
+    "puzzle_kv_amax_update",
+    "puzzle_kv_scales_from_amax",
     "puzzle_kv_append",
     "puzzle_decode_attn_workspace_bytes",
     "puzzle_decode_attn_workspace_init",
@@ -66,6 +68,10 @@ def _load():
         vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
         lib.puzzle_kv_append.restype = ctypes.c_int
         lib.puzzle_kv_append.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, i32, vp, vp]
+        lib.puzzle_kv_amax_update.restype = ctypes.c_int
+        lib.puzzle_kv_amax_update.argtypes = [vp, ctypes.c_int64, i32, i32, vp, vp]
+        lib.puzzle_kv_scales_from_amax.restype = ctypes.c_int
+        lib.puzzle_kv_scales_from_amax.argtypes = [vp, i32, i32, vp, vp]
         lib.puzzle_decode_attn_workspace_bytes.restype = sz
         lib.puzzle_decode_attn_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32, i32]
         lib.puzzle_decode_attn_workspace_init.restype = ctypes.c_int
@@ -156,6 +162,31 @@ def puzzle_kv_append(desc: LayerDesc, view: KVView, k_new: torch.Tensor, v_new: 
     _check(_load().puzzle_kv_append(ctypes.byref(desc), ctypes.byref(view), _p(k_new, torch.bfloat16, "k_new"),
                                     _p(v_new, torch.bfloat16, "v_new"), batch, _p(dev_status, torch.int32),
                                     _stream(stream)), "puzzle_kv_append")
+
+
+def puzzle_kv_amax_update(x: torch.Tensor, amax: torch.Tensor, stream=None) -> None:
+    """x: bf16 [n_tokens][Hkv][D] (any leading dims, flattened); amax: float32 [Hkv], raised in place."""
+    hkv, d = x.shape[-2], x.shape[-1]
+    n_tokens = x.numel() // (hkv * d) if x.numel() else 0
+    _check(_load().puzzle_kv_amax_update(_p(x, torch.bfloat16, "x"), n_tokens, hkv, d, _p(amax, torch.float32, "amax"),
+                                         _stream(stream)), "puzzle_kv_amax_update")
+
+
+def puzzle_kv_scales_from_amax(amax: torch.Tensor, scale_out: torch.Tensor, pow2: bool = False, stream=None) -> None:
+    _check(_load().puzzle_kv_scales_from_amax(_p(amax, torch.float32, "amax"), amax.numel(), int(bool(pow2)),
+                                              _p(scale_out, torch.float32, "scale_out"), _stream(stream)),
+           "puzzle_kv_scales_from_amax")
+
+
+def calibrate_scales(chunks, num_kv_heads: int, pow2: bool = False, device="cuda") -> torch.Tensor:
+    """Max-calibrated scales [num_kv_heads] from an iterable of bf16 tensors [..., Hkv, D] (argument
+    marshalling only: one amax update per chunk, then the quotient)."""
+    amax = torch.zeros(num_kv_heads, dtype=torch.float32, device=device)
+    for x in chunks:
+        puzzle_kv_amax_update(x, amax)
+    scale = torch.empty_like(amax)
+    puzzle_kv_scales_from_amax(amax, scale, pow2)
+    return scale
 
 
 def puzzle_decode_attn_workspace_bytes(desc: LayerDesc, batch: int, num_splits: int = 0) -> int:

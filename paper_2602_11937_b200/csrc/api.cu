@@ -241,6 +241,30 @@ puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_desc* desc, i
                                                                                                   : PUZZLE_ERR_CUDA;
 }
 
+puzzle_status puzzle_kv_amax_update(const void* x, int64_t n_tokens, int32_t num_kv_heads, int32_t head_dim,
+                                    float* amax, void* stream) {
+  if (!amax || (!x && n_tokens > 0)) return PUZZLE_ERR_NULL;
+  if (n_tokens < 0 || num_kv_heads <= 0 || num_kv_heads > calibrate_max_heads() || head_dim <= 0 || head_dim % 8)
+    return PUZZLE_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(amax) & 3)) return PUZZLE_ERR_SHAPE;
+  if (n_tokens == 0) return PUZZLE_OK;
+  if (launch_amax_update(x, n_tokens, num_kv_heads, head_dim, amax, grid_ctas(), static_cast<cudaStream_t>(stream)) !=
+      cudaSuccess)
+    return PUZZLE_ERR_CUDA;
+  count_launch();
+  return PUZZLE_OK;
+}
+
+puzzle_status puzzle_kv_scales_from_amax(const float* amax, int32_t num_kv_heads, int32_t pow2, float* scale_out,
+                                         void* stream) {
+  if (!amax || !scale_out) return PUZZLE_ERR_NULL;
+  if (num_kv_heads <= 0 || num_kv_heads > calibrate_max_heads()) return PUZZLE_ERR_SHAPE;
+  if (launch_scales_from_amax(amax, num_kv_heads, pow2, scale_out, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return PUZZLE_ERR_CUDA;
+  count_launch();
+  return PUZZLE_OK;
+}
+
 puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, const int32_t* num_parts,
                                 const float* sinks, void* out, float* lse_out, int32_t batch, int32_t Hq, int32_t D,
                                 int32_t S, void* stream) {

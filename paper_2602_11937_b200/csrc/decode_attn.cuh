@@ -68,4 +68,10 @@ __global__ void kv_append_kernel(void* k_cache, void* v_cache, const __nv_bfloat
 
 __global__ void hbm_read_probe_kernel(const uint4* buf, size_t n16, unsigned long long* sink);
 
+// Max calibration (calibrate.cu).
+cudaError_t launch_amax_update(const void* x, long long n_tokens, int Hkv, int D, float* amax, int sm_count,
+                               cudaStream_t s);
+cudaError_t launch_scales_from_amax(const float* amax, int Hkv, int pow2, float* scale, cudaStream_t s);
+int calibrate_max_heads();
+
 }  // namespace puzzle
