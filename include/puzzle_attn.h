@@ -173,6 +173,26 @@ PUZZLE_API puzzle_status puzzle_decode_attn_tcgen05(const puzzle_layer_desc* des
                                  int32_t num_splits, void* workspace, size_t workspace_bytes,
                                  int32_t* dev_status, void* stream);
 
+/* This device's share of a decode-step attention whose context is spread over several devices: the
+ * same computation as puzzle_decode_attn over the keys THIS cache view holds, without any sink, with
+ * the result left in float32 for a later merge:
+ *   o_part[b][g][:] = sum_j e^(s_j - lse) v_j,  lse_part[b][g] = ln sum_j e^(s_j),  j over the visible keys
+ * (zeros and -inf when the view holds no visible key).  Every device of a context-sharded layer calls
+ * this on its slice of every sequence (seq_lens = tokens of the slice, its own block table), the
+ * partials are exchanged (one all-gather of batch * Hq * (D + 1) floats per device), and
+ * puzzle_attn_merge_strided applies the sink once.  (Paper: long-context decode is bound by KV-cache
+ * I/O, Section "Optimized Scenarios"; serving sweeps tensor-parallel degree 1..8, paragraph "Inference
+ * efficiency benchmarking"; the 8-GPU 64K/64K study, Section "B200 Inference Efficiency Case Study".
+ * The paper does not describe context sharding itself.)
+ *   o_part: device float32 [batch][Hq][D], 16-byte aligned; lse_part: device float32 [batch][Hq],
+ *   required.  Other arguments, workspace and errors as puzzle_decode_attn.  A window counts back from
+ *   the END of the slice, so a window layer is sharded only if the caller gives each device the window
+ *   that remains on it (the same for every sequence), or keeps window layers on one device. */
+PUZZLE_API puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* desc, const puzzle_kv_view* kv,
+                                 const void* q, float* o_part, float* lse_part, int32_t batch,
+                                 int32_t num_splits, void* workspace, size_t workspace_bytes,
+                                 int32_t* dev_status, void* stream);
+
 /* Size of the scratch array built into the library for puzzle_decode_attn_static. */
 #define PUZZLE_STATIC_SCRATCH_BYTES (8u << 20)
 
@@ -213,6 +233,19 @@ PUZZLE_API puzzle_status puzzle_decode_attn_static(const puzzle_layer_desc* desc
 PUZZLE_API puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, const int32_t* num_parts,
                                 const float* sinks, void* out, float* lse_out, int32_t batch, int32_t Hq,
                                 int32_t D, int32_t S, void* stream);
+
+/* puzzle_attn_merge over partials laid out with strides (in floats): part k of row r = b * Hq + g has
+ * its D outputs at part_o + r * o_row_stride + k * o_part_stride and its lse at
+ * part_lse[r * lse_row_stride + k * lse_part_stride].  An all-gather of per-device buffers
+ * {o [batch][Hq][D], lse [batch][Hq]} is merged in place with o_row_stride = D,
+ * o_part_stride = lse_part_stride = batch * Hq * (D + 1), lse_row_stride = 1 and
+ * part_lse = part_o + batch * Hq * D.  o_row_stride and o_part_stride must be even, no stride negative
+ * (PUZZLE_ERR_SHAPE).  Everything else as puzzle_attn_merge, which is this call with the strides of
+ * a [batch][Hq][S][D] array. */
+PUZZLE_API puzzle_status puzzle_attn_merge_strided(const float* part_o, const float* part_lse, int64_t o_row_stride,
+                                 int64_t o_part_stride, int64_t lse_row_stride, int64_t lse_part_stride,
+                                 const int32_t* num_parts, const float* sinks, void* out, float* lse_out,
+                                 int32_t batch, int32_t Hq, int32_t D, int32_t S, void* stream);
 
 /* Read-only streaming pass over `bytes` bytes at `buf` (16-byte aligned,
  * bytes a multiple of 16): the XOR of all words is written to *sink (device,

@@ -19,7 +19,9 @@ from .binding import (  # noqa: F401
     layer_desc,
     library_path,
     puzzle_attn_merge,
+    puzzle_attn_merge_strided,
     puzzle_decode_attn,
+    puzzle_decode_attn_partial,
     puzzle_decode_attn_static,
     puzzle_decode_attn_tcgen05,
     puzzle_decode_attn_workspace_bytes,
@@ -32,3 +34,4 @@ from .binding import (  # noqa: F401
     puzzle_status_string,
 )
 from .stack import DecodeStack  # noqa: F401,E402
+from .parallel import ContextShardedAttention, context_slice, head_slice  # noqa: F401,E402

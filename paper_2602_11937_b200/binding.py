@@ -28,7 +28,9 @@ EXPORTS = (
     "puzzle_decode_attn",
     "puzzle_decode_attn_tcgen05",
     "puzzle_decode_attn_static",
+    "puzzle_decode_attn_partial",
     "puzzle_attn_merge",
+    "puzzle_attn_merge_strided",
     "puzzle_hbm_read_probe",
     "puzzle_status_string",
     "puzzle_launch_count",
@@ -81,6 +83,12 @@ def _load():
                                            vp, sz, vp, vp]
         lib.puzzle_decode_attn_tcgen05.restype = ctypes.c_int
         lib.puzzle_decode_attn_tcgen05.argtypes = lib.puzzle_decode_attn.argtypes
+        lib.puzzle_decode_attn_partial.restype = ctypes.c_int
+        lib.puzzle_decode_attn_partial.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, i32, i32,
+                                                   vp, sz, vp, vp]
+        lib.puzzle_attn_merge_strided.restype = ctypes.c_int
+        lib.puzzle_attn_merge_strided.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                                  vp, vp, vp, vp, i32, i32, i32, i32, vp]
         lib.puzzle_decode_attn_static.restype = ctypes.c_int
         lib.puzzle_decode_attn_static.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp,
                                                   i32, i32, vp, vp]
@@ -238,6 +246,34 @@ def puzzle_decode_attn_static(desc: LayerDesc, view: KVView, q: torch.Tensor, si
                                              _p(lse_out, torch.float32, "lse_out"), q.shape[0], int(num_splits),
                                              _p(dev_status, torch.int32), _stream(stream)),
            "puzzle_decode_attn_static")
+
+
+def puzzle_decode_attn_partial(desc: LayerDesc, view: KVView, q: torch.Tensor, o_part: torch.Tensor,
+                               lse_part: torch.Tensor, num_splits: int = 0, workspace: Optional[torch.Tensor] = None,
+                               dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """This device's float32 partial (o, lse) over the keys its view holds, no sink: see the header."""
+    if workspace is None:
+        raise ValueError("workspace is required (size it with puzzle_decode_attn_workspace_bytes)")
+    _check(_load().puzzle_decode_attn_partial(ctypes.byref(desc), ctypes.byref(view), _p(q, torch.bfloat16, "q"),
+                                              _p(o_part, torch.float32, "o_part"),
+                                              _p(lse_part, torch.float32, "lse_part"), q.shape[0], int(num_splits),
+                                              _p(workspace), workspace.numel() * workspace.element_size(),
+                                              _p(dev_status, torch.int32), _stream(stream)),
+           "puzzle_decode_attn_partial")
+
+
+def puzzle_attn_merge_strided(part_o: torch.Tensor, part_lse: torch.Tensor, o_row_stride: int, o_part_stride: int,
+                              lse_row_stride: int, lse_part_stride: int, num_parts: Optional[torch.Tensor],
+                              sinks: Optional[torch.Tensor], out: torch.Tensor, num_parts_max: int,
+                              lse_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """part_o / part_lse: float32 tensors whose first elements are part 0 of row 0 (strides in floats)."""
+    batch, hq, d = out.shape
+    _check(_load().puzzle_attn_merge_strided(_p(part_o, torch.float32, "part_o"), _p(part_lse, torch.float32, "part_lse"),
+                                             int(o_row_stride), int(o_part_stride), int(lse_row_stride),
+                                             int(lse_part_stride), _p(num_parts, torch.int32, "num_parts"),
+                                             _p(sinks, torch.float32, "sinks"), _p(out, torch.bfloat16, "out"),
+                                             _p(lse_out, torch.float32, "lse_out"), batch, hq, d, int(num_parts_max),
+                                             _stream(stream)), "puzzle_attn_merge_strided")
 
 
 def puzzle_attn_merge(part_o: torch.Tensor, part_lse: torch.Tensor, num_parts: Optional[torch.Tensor],

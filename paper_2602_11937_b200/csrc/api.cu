@@ -152,7 +152,7 @@ size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t
 static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
                                       const float* sinks, void* out, float* lse_out, int32_t batch,
                                       int32_t num_splits, void* workspace, size_t workspace_bytes,
-                                      int32_t* dev_status, void* stream, bool tcgen05) {
+                                      int32_t* dev_status, void* stream, bool tcgen05, bool out_f32 = false) {
   puzzle_status st = check_desc(desc);
   if (st != PUZZLE_OK) return st;
   st = check_view(desc, kv, batch);
@@ -193,7 +193,8 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   P.part_lse = part_lse;
   P.counters = static_cast<int32_t*>(workspace);
   P.sinks = sinks;
-  P.out = static_cast<__nv_bfloat16*>(out);
+  P.out = out_f32 ? nullptr : static_cast<__nv_bfloat16*>(out);
+  P.out_f32 = out_f32 ? static_cast<float*>(out) : nullptr;
   P.lse_out = lse_out;
   P.dev_status = dev_status;
   P.num_blocks = kv->num_blocks;
@@ -227,6 +228,15 @@ puzzle_status puzzle_decode_attn_tcgen05(const puzzle_layer_desc* desc, const pu
                                          int32_t* dev_status, void* stream) {
   return decode_attn_impl(desc, kv, q, sinks, out, lse_out, batch, num_splits, workspace, workspace_bytes, dev_status,
                           stream, true);
+}
+
+puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                         float* o_part, float* lse_part, int32_t batch, int32_t num_splits,
+                                         void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                         void* stream) {
+  if (!lse_part) return PUZZLE_ERR_NULL;
+  return decode_attn_impl(desc, kv, q, nullptr, o_part, lse_part, batch, num_splits, workspace, workspace_bytes,
+                          dev_status, stream, false, true);
 }
 
 puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_desc* desc, int32_t batch, void* workspace,
@@ -265,17 +275,25 @@ puzzle_status puzzle_kv_scales_from_amax(const float* amax, int32_t num_kv_heads
   return PUZZLE_OK;
 }
 
-puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, const int32_t* num_parts,
-                                const float* sinks, void* out, float* lse_out, int32_t batch, int32_t Hq, int32_t D,
-                                int32_t S, void* stream) {
+puzzle_status puzzle_attn_merge_strided(const float* part_o, const float* part_lse, int64_t o_row_stride,
+                                        int64_t o_part_stride, int64_t lse_row_stride, int64_t lse_part_stride,
+                                        const int32_t* num_parts, const float* sinks, void* out, float* lse_out,
+                                        int32_t batch, int32_t Hq, int32_t D, int32_t S, void* stream) {
   if (!part_o || !part_lse || !out) return PUZZLE_ERR_NULL;
   if (batch <= 0 || Hq <= 0 || S <= 0 || D <= 0) return PUZZLE_ERR_SHAPE;
   if (D % 64 != 0 || D > 512) return PUZZLE_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(part_o) & 7) || (reinterpret_cast<uintptr_t>(out) & 3)) return PUZZLE_ERR_SHAPE;
+  if (o_row_stride < 0 || o_part_stride < 0 || lse_row_stride < 0 || lse_part_stride < 0 || (o_row_stride & 1) ||
+      (o_part_stride & 1))
+    return PUZZLE_ERR_SHAPE;   // partial rows are read two floats at a time
   MergeParams M;
   std::memset(&M, 0, sizeof M);
   M.part_o = part_o;
   M.part_lse = part_lse;
+  M.o_row_stride = o_row_stride;
+  M.o_part_stride = o_part_stride;
+  M.lse_row_stride = lse_row_stride;
+  M.lse_part_stride = lse_part_stride;
   M.num_parts = num_parts;
   M.sinks = sinks;
   M.out = static_cast<__nv_bfloat16*>(out);
@@ -288,6 +306,13 @@ puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, cons
   attn_merge_kernel<<<(unsigned)((rows + kWarps - 1) / kWarps), kWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(M);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+}
+
+puzzle_status puzzle_attn_merge(const float* part_o, const float* part_lse, const int32_t* num_parts,
+                                const float* sinks, void* out, float* lse_out, int32_t batch, int32_t Hq, int32_t D,
+                                int32_t S, void* stream) {
+  return puzzle_attn_merge_strided(part_o, part_lse, (int64_t)S * D, D, S, 1, num_parts, sinks, out, lse_out, batch, Hq,
+                                   D, S, stream);
 }
 
 puzzle_status puzzle_hbm_read_probe(const void* buf, size_t bytes, uint64_t* sink, void* stream) {

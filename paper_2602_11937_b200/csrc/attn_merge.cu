@@ -12,13 +12,13 @@ __global__ void __launch_bounds__(kWarps * 32) attn_merge_kernel(const MergePara
   const long long row = (long long)blockIdx.x * kWarps + warp;
   if (row >= (long long)P.batch * P.Hq) return;
   const int b = (int)(row / P.Hq), head = (int)(row % P.Hq);
-  const long long first = row * P.S;
+  const float* lse_row = P.part_lse + row * P.lse_row_stride;
+  const float* o_row = P.part_o + row * P.o_row_stride;
   const int count = P.num_parts ? min(max(P.num_parts[b], 0), P.S) : P.S;
-  const int stride = 1;
 
   const float sink = P.sinks ? P.sinks[head] : -INFINITY;
   float M = sink;
-  for (int k = lane; k < count; k += 32) M = fmaxf(M, P.part_lse[first + (long long)k * stride]);
+  for (int k = lane; k < count; k += 32) M = fmaxf(M, lse_row[k * P.lse_part_stride]);
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
 
@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_merge_kernel(const MergePara
   }
   float Z = 0.f;
   for (int k = lane; k < count; k += 32) {
-    const float l = P.part_lse[first + (long long)k * stride];
+    const float l = lse_row[k * P.lse_part_stride];
     if (l != -INFINITY) Z += __expf(l - M);
   }
 #pragma unroll
@@ -41,11 +41,10 @@ __global__ void __launch_bounds__(kWarps * 32) attn_merge_kernel(const MergePara
   for (int d = 2 * lane; d < P.D; d += 64) {
     float ax = 0.f, ay = 0.f;
     for (int k = 0; k < count; ++k) {
-      const long long idx = first + (long long)k * stride;
-      const float l = P.part_lse[idx];
+      const float l = lse_row[k * P.lse_part_stride];
       if (l == -INFINITY) continue;
       const float wgt = __expf(l - M);
-      const float2 o = *reinterpret_cast<const float2*>(P.part_o + idx * P.D + d);
+      const float2 o = *reinterpret_cast<const float2*>(o_row + k * P.o_part_stride + d);
       ax += wgt * o.x;
       ay += wgt * o.y;
     }

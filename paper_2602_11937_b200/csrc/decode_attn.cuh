@@ -21,6 +21,7 @@ struct alignas(64) DecodeParams {
   int32_t* counters;   // [batch*Hkv] arrivals per (sequence, KV head); zero before and after every launch
   const float* sinks;  // [Hq] or null
   __nv_bfloat16* out;  // [batch][Hq][D]
+  float* out_f32;      // when set, the merged rows are stored here as float32 instead (out is unused)
   float* lse_out;      // [batch][Hq] or null
   int32_t* dev_status;
   long long num_blocks;
@@ -32,8 +33,9 @@ struct alignas(64) DecodeParams {
 };
 
 struct MergeParams {
-  const float* part_o;       // [rows][S][D]
-  const float* part_lse;     // [rows][S]
+  const float* part_o;       // part k of row r starts at part_o + r * o_row_stride + k * o_part_stride
+  const float* part_lse;     // part k of row r is part_lse[r * lse_row_stride + k * lse_part_stride]
+  long long o_row_stride, o_part_stride, lse_row_stride, lse_part_stride;   // in floats
   const int32_t* num_parts;  // [batch] or null
   const float* sinks;
   __nv_bfloat16* out;

@@ -122,12 +122,19 @@ __device__ __noinline__ void merge_rows(const DecodeParams& P, int b, int kvh, l
     if (sink != -INFINITY) Z += __expf(sink - M);  // the sink is one more softmax column, counted once
   }
   const float invZ = Z > 0.f ? 1.f / Z : 0.f;  // nothing visible and no sink: zeros
-  uint32_t packed[8];
+  if (P.out_f32) {  // a partial for a merge across devices keeps float32
+    float4* dst = reinterpret_cast<float4*>(P.out_f32 + row_out * kHeadDim + 16 * c);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) packed[i] = f32x2_to_bf16x2(acc[2 * i] * invZ, acc[2 * i + 1] * invZ);
-  uint4* dst = reinterpret_cast<uint4*>(P.out + row_out * kHeadDim + 16 * c);
-  dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-  dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+    for (int i = 0; i < 4; ++i)
+      dst[i] = make_float4(acc[4 * i] * invZ, acc[4 * i + 1] * invZ, acc[4 * i + 2] * invZ, acc[4 * i + 3] * invZ);
+  } else {
+    uint32_t packed[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) packed[i] = f32x2_to_bf16x2(acc[2 * i] * invZ, acc[2 * i + 1] * invZ);
+    uint4* dst = reinterpret_cast<uint4*>(P.out + row_out * kHeadDim + 16 * c);
+    dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+  }
   if (P.lse_out && c == 0) P.lse_out[row_out] = Z > 0.f ? M + __logf(Z) : -INFINITY;
 }
 
