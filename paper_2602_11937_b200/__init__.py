@@ -34,4 +34,5 @@ from .binding import (  # noqa: F401
     puzzle_status_string,
 )
 from .stack import DecodeStack  # noqa: F401,E402
+from .paging import cache_blocks, linear_block_table, ring_block_table, window_ring_blocks  # noqa: F401,E402
 from .parallel import ContextShardedAttention, context_slice, head_slice  # noqa: F401,E402

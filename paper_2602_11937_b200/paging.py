@@ -1,0 +1,44 @@
+"""Block tables for the paged KV cache (host-side index arithmetic only).
+
+A window layer attends to the W most recent tokens, so it never needs more than ``ceil(W / 16) + 1`` blocks of a
+sequence at a time: that is where the paper's KV-cache saving comes from (window layers keep a bounded cache,
+Section "Window attention for long-context inference"; a 40 % smaller KV cache in the 64K scenario, Section
+"Optimized Scenarios").  The kernels read a block only through the table and never look at entries wholly
+before the window, so the saving needs no kernel support: a window layer's table maps logical block ``j`` of a
+sequence onto a ring of ``R`` physical blocks, ``j % R``.  The append of token ``L - 1`` then overwrites the
+block that left the window ``R`` blocks ago.
+"""
+from __future__ import annotations
+
+import torch
+
+BLOCK = 16
+
+
+def window_ring_blocks(window: int, block: int = BLOCK) -> int:
+    """Physical blocks per sequence that a layer with this window needs (window >= 1)."""
+    if window < 1:
+        raise ValueError("a full-attention layer keeps every block")
+    return (window + block - 1) // block + 1
+
+
+def ring_block_table(batch: int, window: int, max_blocks_per_seq: int, first_block: int = 0, block: int = BLOCK,
+                     device="cpu") -> torch.Tensor:
+    """int32 [batch][max_blocks_per_seq] table of a window layer whose sequence b owns the physical blocks
+    ``first_block + b * R .. + R - 1``, R = window_ring_blocks(window): logical block j -> ring slot j % R."""
+    r = window_ring_blocks(window, block)
+    j = torch.arange(max_blocks_per_seq, dtype=torch.int64, device=device)[None, :] % r
+    b = torch.arange(batch, dtype=torch.int64, device=device)[:, None] * r
+    return (first_block + b + j).to(torch.int32)
+
+
+def linear_block_table(batch: int, max_blocks_per_seq: int, first_block: int = 0, device="cpu") -> torch.Tensor:
+    """The table of a full-attention layer with one private run of blocks per sequence."""
+    j = torch.arange(max_blocks_per_seq, dtype=torch.int64, device=device)[None, :]
+    b = torch.arange(batch, dtype=torch.int64, device=device)[:, None] * max_blocks_per_seq
+    return (first_block + b + j).to(torch.int32)
+
+
+def cache_blocks(windows, batch: int, max_blocks_per_seq: int) -> list:
+    """Physical blocks each layer of a stack needs: all of them for full layers (window 0), a ring for the rest."""
+    return [batch * (max_blocks_per_seq if w == 0 else min(max_blocks_per_seq, window_ring_blocks(w))) for w in windows]

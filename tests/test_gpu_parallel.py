@@ -102,8 +102,9 @@ def test_kv_head_sharding_needs_no_exchange(world):
     for r in range(world):
         kvs, qs = head_slice(r, world, w.hkv, w.hq // w.hkv)
         kc, vc = dev.k_cache[:, kvs].contiguous(), dev.v_cache[:, kvs].contiguous()
+        ksc, vsc = dev.k_scale[kvs].contiguous(), dev.v_scale[kvs].contiguous()   # the view keeps raw pointers
         view = P.kv_view(kc, vc, dev.seq_lens, block_table=dev.table, max_blocks_per_seq=w.blocks_per_seq,
-                         k_scale=dev.k_scale[kvs].contiguous(), v_scale=dev.v_scale[kvs].contiguous())
+                         k_scale=ksc, v_scale=vsc)
         d = P.layer_desc(window=0, num_q_heads=w.hq // world, num_kv_heads=w.hkv // world)
         ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(d, w.batch, 0), dtype=torch.uint8, device="cuda")
         P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
