@@ -37,9 +37,20 @@ __global__ void __launch_bounds__(kCalThreads) amax_update_kernel(const uint4* _
   // A thread keeps the maximum of the head it is looking at in a register and hands it to shared memory when
   // the head changes; with a stride that is a multiple of one token's chunks the head never changes.
   const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long start = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   int head = -1;
   uint32_t m = 0;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_chunks; i += stride) {
+  long long i = start;
+  if (stride % ((long long)chunks_per_head_row * Hkv) == 0 && start < n_chunks) {
+    // the common case: one head per thread for the whole pass, four independent loads per round
+    head = (int)((start / chunks_per_head_row) % Hkv);
+    for (; i + 3 * stride < n_chunks; i += 4 * stride) {
+      const uint4 a = __ldcs(x + i), b = __ldcs(x + i + stride), c = __ldcs(x + i + 2 * stride),
+                  d = __ldcs(x + i + 3 * stride);
+      m = max(max(m, chunk_amax_bits(a)), max(chunk_amax_bits(b), max(chunk_amax_bits(c), chunk_amax_bits(d))));
+    }
+  }
+  for (; i < n_chunks; i += stride) {
     const int h = (int)((i / chunks_per_head_row) % Hkv);
     if (h != head) {
       if (head >= 0 && m) atomicMax(&s_amax[head], m);
