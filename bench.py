@@ -185,11 +185,19 @@ def run_ours(args):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
-    def step(i):
+    attn_events = []   # CUDA-event pairs around the attention launch of every 8th timed step
+
+    def step(i, sample=False):
         v = views[i % len(views)]
         P.puzzle_kv_append(desc, v, k_new, v_new, dev_status=status, stream=stream)
+        if sample:
+            ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ea.record(stream)
         decode(desc, v, q, sinks, out, None, num_splits=args.splits, workspace=ws,
                              dev_status=status, stream=stream)
+        if sample:
+            eb.record(stream)
+            attn_events.append((ea, eb))
 
     def barrier():
         if world > 1:
@@ -209,11 +217,12 @@ def run_ours(args):
     barrier()
     t0.record(stream)
     for i in range(args.steps):
-        step(i)
+        step(i, sample=(i % 8 == 7))
     t1.record(stream)
     barrier()
     launches = P.puzzle_launch_count() - launches0
     ms_total = t0.elapsed_time(t1)
+    attn_in_region_ms = [a.elapsed_time(b) for a, b in attn_events]
     # the attention kernel alone: the same launches back to back on the same stream, no append in between
     n_attn = min(args.steps, 400)
     a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -270,7 +279,11 @@ def run_ours(args):
     dev_flags = int(status.item())
     bytes_step = algorithmic_bytes(w, seq_lens_host, window)
     kv_bytes_attn = bytes_step - 2 * w.batch * w.hkv * w.head_dim * 3   # what the attention pass itself moves
-    ms_total, ms_e2e, attn_mean_ms = max_over_ranks([ms_total, ms_e2e, statistics.mean(attn_ms)], world, dev)
+    # roofline: mean duration of the attention launches sampled INSIDE the timed region (falls back to the
+    # back-to-back loop when the run is too short to hold a sample)
+    b2b_ms = statistics.mean(attn_ms)
+    in_region_ms = statistics.mean(attn_in_region_ms) if attn_in_region_ms else b2b_ms
+    ms_total, ms_e2e, attn_mean_ms, b2b_ms = max_over_ranks([ms_total, ms_e2e, in_region_ms, b2b_ms], world, dev)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -298,7 +311,8 @@ def run_ours(args):
                          "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
                          "unit": "GB/s", "frac": round(achieved / peak, 4),
                          "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
-                         "us_per_launch": round(attn_mean_ms * 1e3, 2), "bytes_per_launch": int(kv_bytes_attn),
+                         "us_per_launch": round(attn_mean_ms * 1e3, 2), "launches_sampled": len(attn_in_region_ms),
+                         "us_per_launch_back_to_back": round(b2b_ms * 1e3, 2), "bytes_per_launch": int(kv_bytes_attn),
                          "read_probe_gbs": round(probe_gbs, 1),
                          "traffic": ncu_traffic(args)},
             "dev_status": dev_flags,

@@ -119,6 +119,19 @@ PUZZLE_API puzzle_status puzzle_kv_scales_from_amax(const float* amax, int32_t n
 PUZZLE_API puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* k_new,
                                const void* v_new, int32_t batch, int32_t* dev_status, void* stream);
 
+/* puzzle_kv_append for n_new tokens per sequence at once: a chunk of the prompt, or the tokens of a
+ * multi-token decode step (the input half of the paper's fixed-length scenarios, Section "Optimized
+ * Scenarios"; same quantisation, Section "KV Quantization").  Token i of sequence b lands at logical
+ * position seq_lens[b] - new_lens[b] + i, seq_lens counted AFTER the append.
+ *   k_new, v_new: device bf16 [batch][n_new][num_kv_heads][head_dim], 16-byte aligned;
+ *   new_lens: device int32 [batch], tokens of each row that are real (clamped to [0, n_new]; the rest of
+ *     the row is ignored), or NULL = n_new for every sequence.  Tokens that would land before position
+ *     0 (new_lens[b] > seq_lens[b]) are skipped.
+ * Errors and dev_status as puzzle_kv_append. */
+PUZZLE_API puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, const puzzle_kv_view* kv,
+                                 const void* k_new, const void* v_new, const int32_t* new_lens, int32_t batch,
+                                 int32_t n_new, int32_t* dev_status, void* stream);
+
 /* Bytes of scratch puzzle_decode_attn needs for this batch and split choice
  * (0 on invalid arguments).  num_splits == 0 selects the balanced schedule. */
 PUZZLE_API size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits);

@@ -29,10 +29,11 @@ from .binding import (  # noqa: F401
     puzzle_hbm_read_probe,
     puzzle_kv_amax_update,
     puzzle_kv_append,
+    puzzle_kv_append_tokens,
     puzzle_kv_scales_from_amax,
     puzzle_launch_count,
     puzzle_status_string,
 )
 from .stack import DecodeStack  # noqa: F401,E402
-from .paging import cache_blocks, linear_block_table, ring_block_table, window_ring_blocks  # noqa: F401,E402
+from .paging import cache_blocks, linear_block_table, multi_token_args, ring_block_table, window_ring_blocks  # noqa: F401,E402
 from .parallel import ContextShardedAttention, context_slice, head_slice  # noqa: F401,E402

@@ -23,6 +23,7 @@ EXPORTS = (
     "puzzle_kv_amax_update",
     "puzzle_kv_scales_from_amax",
     "puzzle_kv_append",
+    "puzzle_kv_append_tokens",
     "puzzle_decode_attn_workspace_bytes",
     "puzzle_decode_attn_workspace_init",
     "puzzle_decode_attn",
@@ -74,6 +75,9 @@ def _load():
         lib.puzzle_kv_amax_update.argtypes = [vp, ctypes.c_int64, i32, i32, vp, vp]
         lib.puzzle_kv_scales_from_amax.restype = ctypes.c_int
         lib.puzzle_kv_scales_from_amax.argtypes = [vp, i32, i32, vp, vp]
+        lib.puzzle_kv_append_tokens.restype = ctypes.c_int
+        lib.puzzle_kv_append_tokens.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, i32, i32,
+                                                vp, vp]
         lib.puzzle_decode_attn_workspace_bytes.restype = sz
         lib.puzzle_decode_attn_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32, i32]
         lib.puzzle_decode_attn_workspace_init.restype = ctypes.c_int
@@ -195,6 +199,17 @@ def calibrate_scales(chunks, num_kv_heads: int, pow2: bool = False, device="cuda
     scale = torch.empty_like(amax)
     puzzle_kv_scales_from_amax(amax, scale, pow2)
     return scale
+
+
+def puzzle_kv_append_tokens(desc: LayerDesc, view: KVView, k_new: torch.Tensor, v_new: torch.Tensor,
+                            new_lens: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                            stream=None) -> None:
+    """k_new, v_new: bf16 [batch][n_new][Hkv][D]; new_lens: int32 [batch] or None (all n_new tokens are real)."""
+    batch, n_new = k_new.shape[0], k_new.shape[1]
+    _check(_load().puzzle_kv_append_tokens(ctypes.byref(desc), ctypes.byref(view), _p(k_new, torch.bfloat16, "k_new"),
+                                           _p(v_new, torch.bfloat16, "v_new"), _p(new_lens, torch.int32, "new_lens"),
+                                           batch, n_new, _p(dev_status, torch.int32), _stream(stream)),
+           "puzzle_kv_append_tokens")
 
 
 def puzzle_decode_attn_workspace_bytes(desc: LayerDesc, batch: int, num_splits: int = 0) -> int:

@@ -143,6 +143,26 @@ puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_vi
   return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
 }
 
+puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* k_new,
+                                      const void* v_new, const int32_t* new_lens, int32_t batch, int32_t n_new,
+                                      int32_t* dev_status, void* stream) {
+  puzzle_status st = check_desc(desc);
+  if (st != PUZZLE_OK) return st;
+  st = check_view(desc, kv, batch);
+  if (st != PUZZLE_OK) return st;
+  if (!k_new || !v_new) return PUZZLE_ERR_NULL;
+  if (n_new <= 0 || n_new > (1 << 20)) return PUZZLE_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(k_new) & 15) || (reinterpret_cast<uintptr_t>(v_new) & 15)) return PUZZLE_ERR_SHAPE;
+  const long long threads = 2ll * batch * n_new * desc->num_kv_heads * (kHeadDim / 8);
+  if (threads > 0x7fffffffll * 256) return PUZZLE_ERR_SHAPE;
+  kv_append_tokens_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      kv->k_cache, kv->v_cache, static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), new_lens,
+      kv->block_table, kv->seq_lens, kv->k_scale, kv->v_scale, kv->num_blocks, batch, n_new, desc->num_kv_heads,
+      kv->max_blocks_per_seq, desc->kv_dtype, dev_status);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+}
+
 size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits) {
   if (check_desc(desc) != PUZZLE_OK || batch <= 0 || batch > kMaxBatch || num_splits < 0) return 0;
   return counter_bytes(batch, desc->num_kv_heads) +

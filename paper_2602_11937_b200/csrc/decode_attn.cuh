@@ -68,6 +68,10 @@ __global__ void kv_append_kernel(void* k_cache, void* v_cache, const __nv_bfloat
                                  const float* k_scale, const float* v_scale, long long num_blocks, int batch, int Hkv,
                                  int max_blocks_per_seq, int kv_dtype, int32_t* dev_status);
 
+__global__ void kv_append_tokens_kernel(void* k_cache, void* v_cache, const uint4* k_new, const uint4* v_new,
+                                        const int32_t* new_lens, const int32_t* block_table, const int32_t* seq_lens,
+                                        const float* k_scale, const float* v_scale, long long num_blocks, int batch,
+                                        int n_new, int Hkv, int max_blocks_per_seq, int kv_dtype, int32_t* dev_status);
 __global__ void hbm_read_probe_kernel(const uint4* buf, size_t n16, unsigned long long* sink);
 
 // Max calibration (calibrate.cu).

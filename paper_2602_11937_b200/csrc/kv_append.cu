@@ -58,6 +58,59 @@ __global__ void __launch_bounds__(256) kv_append_kernel(void* k_cache, void* v_c
   }
 }
 
+// Bulk form: n_new tokens per sequence (a prompt chunk, or several tokens of a multi-token step).  Token i of
+// sequence b goes to position seq_lens[b] - new_lens[b] + i (seq_lens counted after the append).  One thread
+// converts eight adjacent channels: a 16-byte load, an 8-byte (FP8) or 16-byte (bf16) store.
+__global__ void __launch_bounds__(256) kv_append_tokens_kernel(void* k_cache, void* v_cache, const uint4* k_new,
+                                                               const uint4* v_new, const int32_t* new_lens,
+                                                               const int32_t* block_table, const int32_t* seq_lens,
+                                                               const float* k_scale, const float* v_scale,
+                                                               long long num_blocks, int batch, int n_new, int Hkv,
+                                                               int max_blocks_per_seq, int kv_dtype,
+                                                               int32_t* dev_status) {
+  constexpr int kOct = kHeadDim / 8;   // 16-byte pieces per (token, head) row
+  const long long per_tensor = (long long)batch * n_new * Hkv * kOct;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= 2 * per_tensor) return;
+  const bool is_v = idx >= per_tensor;
+  const long long i = is_v ? idx - per_tensor : idx;
+  const int o = (int)(i % kOct);
+  const int h = (int)((i / kOct) % Hkv);
+  const int tok = (int)((i / ((long long)kOct * Hkv)) % n_new);
+  const int b = (int)(i / ((long long)kOct * Hkv * n_new));
+
+  const int len = seq_lens[b];
+  const int nl = new_lens ? min(max(new_lens[b], 0), n_new) : n_new;
+  const bool reporter = o == 0 && h == 0 && tok == 0 && !is_v;
+  if (len > max_blocks_per_seq * kBlock) {
+    if (dev_status && reporter) atomicOr(dev_status, (int)PUZZLE_DEV_SEQ_TOO_LONG);
+    return;
+  }
+  const int pos = len - nl + tok;
+  if (tok >= nl || pos < 0) return;   // a sequence shorter than its chunk keeps the chunk's last `len` tokens
+  const long long blk = block_table ? (long long)block_table[(size_t)b * max_blocks_per_seq + pos / kBlock]
+                                    : (long long)b * max_blocks_per_seq + pos / kBlock;
+  if (blk < 0 || blk >= num_blocks) {
+    if (dev_status && o == 0 && h == 0 && !is_v) atomicOr(dev_status, (int)PUZZLE_DEV_BAD_BLOCK);
+    return;
+  }
+  const size_t dst = ((size_t)(blk * Hkv + h) * kBlock + pos % kBlock) * kHeadDim + 8 * o;   // in elements
+  const uint4 x = __ldcs((is_v ? v_new : k_new) + i);
+  void* cache = is_v ? v_cache : k_cache;
+  if (kv_dtype == PUZZLE_KV_BF16) {
+    reinterpret_cast<uint4*>(cache)[dst / 8] = x;
+  } else {
+    const float* sp = is_v ? v_scale : k_scale;
+    const float s = sp ? sp[h] : 1.f;
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+    uint32_t c[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      c[k] = encode_e4m3_pair(__fdiv_rn(__uint_as_float(w[k] << 16), s), __fdiv_rn(__uint_as_float(w[k] & 0xffff0000u), s));
+    reinterpret_cast<uint2*>(cache)[dst / 8] = make_uint2((c[0] & 0xffffu) | (c[1] << 16), (c[2] & 0xffffu) | (c[3] << 16));
+  }
+}
+
 // Read-only streaming probe: XOR-reduces the buffer so the loads cannot be dropped.
 __global__ void __launch_bounds__(512) hbm_read_probe_kernel(const uint4* buf, size_t n16, unsigned long long* sink) {
   uint4 acc = make_uint4(0, 0, 0, 0);

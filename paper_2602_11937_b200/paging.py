@@ -42,3 +42,29 @@ def linear_block_table(batch: int, max_blocks_per_seq: int, first_block: int = 0
 def cache_blocks(windows, batch: int, max_blocks_per_seq: int) -> list:
     """Physical blocks each layer of a stack needs: all of them for full layers (window 0), a ring for the rest."""
     return [batch * (max_blocks_per_seq if w == 0 else min(max_blocks_per_seq, window_ring_blocks(w))) for w in windows]
+
+
+def multi_token_args(seq_lens: torch.Tensor, block_table, n_q: int, max_blocks_per_seq: int = None, q_lens=None):
+    """Arguments that make the decode kernels serve ``n_q`` query tokens per sequence with a causal mask (several
+    tokens of a multi-token step, or a prompt chunk after its bulk append): query row i of sequence b sits at position
+    ``seq_lens[b] - q_lens[b] + i`` and sees the keys up to and including itself, i.e. it is a decode step of a
+    sequence of length ``seq_lens[b] - q_lens[b] + i + 1`` over the same blocks (a window layer then counts back from
+    that position).  Returns ``(lens, table)`` for a batch of ``batch * n_q`` rows: int32 ``[batch * n_q]`` and int32
+    ``[batch * n_q][max_blocks_per_seq]`` (each table row repeated ``n_q`` times).  Rows ``i >= q_lens[b]`` are
+    padding and get length 0 (output 0).  Pass q as ``[batch * n_q][Hq][D]``.
+
+    The n_q rows of a sequence read the same cache blocks at about the same time (they are neighbours in the
+    balanced schedule), so the repeats are served by L2 rather than HBM."""
+    batch = seq_lens.shape[0]
+    dev = seq_lens.device
+    L = seq_lens.to(torch.int64)[:, None]
+    ql = torch.full((batch, 1), n_q, dtype=torch.int64, device=dev) if q_lens is None else \
+        torch.clamp(q_lens.to(torch.int64), 0, n_q)[:, None]
+    i = torch.arange(n_q, dtype=torch.int64, device=dev)[None, :]
+    lens = torch.where(i < ql, torch.clamp(L - ql + i + 1, min=0), torch.zeros_like(i))
+    if block_table is None:
+        if max_blocks_per_seq is None:
+            raise ValueError("max_blocks_per_seq is required without a block table")
+        block_table = linear_block_table(batch, max_blocks_per_seq, device=dev)
+    table = block_table.repeat_interleave(n_q, dim=0).contiguous()
+    return lens.reshape(-1).to(torch.int32).contiguous(), table
