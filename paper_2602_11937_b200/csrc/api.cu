@@ -153,9 +153,10 @@ puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, const puzzl
   if (!k_new || !v_new) return PUZZLE_ERR_NULL;
   if (n_new <= 0 || n_new > (1 << 20)) return PUZZLE_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(k_new) & 15) || (reinterpret_cast<uintptr_t>(v_new) & 15)) return PUZZLE_ERR_SHAPE;
-  const long long threads = 2ll * batch * n_new * desc->num_kv_heads * (kHeadDim / 8);
-  if (threads > 0x7fffffffll * 256) return PUZZLE_ERR_SHAPE;
-  kv_append_tokens_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+  const long long per_seq = (long long)n_new * desc->num_kv_heads * (kHeadDim / 8);
+  if (per_seq > 0x7fffffffll || batch > 65535) return PUZZLE_ERR_SHAPE;
+  const dim3 grid((unsigned)((per_seq + 255) / 256), (unsigned)batch, 2);
+  kv_append_tokens_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
       kv->k_cache, kv->v_cache, static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), new_lens,
       kv->block_table, kv->seq_lens, kv->k_scale, kv->v_scale, kv->num_blocks, batch, n_new, desc->num_kv_heads,
       kv->max_blocks_per_seq, desc->kv_dtype, dev_status);

@@ -69,15 +69,18 @@ __global__ void __launch_bounds__(256) kv_append_tokens_kernel(void* k_cache, vo
                                                                int max_blocks_per_seq, int kv_dtype,
                                                                int32_t* dev_status) {
   constexpr int kOct = kHeadDim / 8;   // 16-byte pieces per (token, head) row
-  const long long per_tensor = (long long)batch * n_new * Hkv * kOct;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= 2 * per_tensor) return;
-  const bool is_v = idx >= per_tensor;
-  const long long i = is_v ? idx - per_tensor : idx;
-  const int o = (int)(i % kOct);
-  const int h = (int)((i / kOct) % Hkv);
-  const int tok = (int)((i / ((long long)kOct * Hkv)) % n_new);
-  const int b = (int)(i / ((long long)kOct * Hkv * n_new));
+  // grid: x over the (token, head, piece) of one sequence, y = sequence, z = K or V
+  const int per_seq = n_new * Hkv * kOct;
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= per_seq) return;
+  const int b = blockIdx.y;
+  const bool is_v = blockIdx.z != 0;
+  // piece fastest, then token, then head: a warp reads four 128-byte head rows and writes 256 contiguous bytes
+  // of one cache block (FP8), so both sides move whole lines
+  const int o = r % kOct;
+  const int tok = (r / kOct) % n_new;
+  const int h = r / (kOct * n_new);
+  const long long i = (((long long)b * n_new + tok) * Hkv + h) * kOct + o;   // 16-byte piece of k_new / v_new
 
   const int len = seq_lens[b];
   const int nl = new_lens ? min(max(new_lens[b], 0), n_new) : n_new;
