@@ -357,8 +357,8 @@ def cpu_baseline(w, layer, seq_lens_host, q, sinks, window, pairs: int = 128):
 NCU_CAPTURE = {
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn.cu", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "ac9e91c4b26adddbbc1a3f1c79630cd5195d13da7ddd13c0d80688a55bbcc52a",
-    "dram_bytes_per_launch": 1075438000 + 4268800,
+    "sha256": "873e8bdb34f774246fe23020f541aa43a28396e833d6749ec2ac0a2eacc17402",
+    "dram_bytes_per_launch": 1075619000 + 4381952,
 }
 
 
