@@ -236,13 +236,18 @@ def run_ours(args):
     clocks = sampler.stop()
 
     # ---- end to end: the step's inputs start in pinned host memory, the result ends there
-    hq_, hk_, hv_ = (t.cpu().pin_memory() for t in (q, k_new, v_new))
+    # q, k_new and v_new of a step travel as ONE pinned host buffer and one copy (the caller's side of the API:
+    # the entry points take three pointers, which may point into one allocation)
+    parts = (q, k_new, v_new)
+    sizes = [t.numel() for t in parts]
+    hin = torch.cat([t.reshape(-1).cpu() for t in parts]).pin_memory()
+    din = torch.empty(sum(sizes), dtype=q.dtype, device=dev)
+    dq, dk, dv = (din[sum(sizes[:k]):sum(sizes[:k + 1])].view(parts[k].shape) for k in range(3))
     hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-    dq, dk, dv = torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new)
 
     def step_e2e(i):
         v = views[i % len(views)]
-        dq.copy_(hq_, non_blocking=True); dk.copy_(hk_, non_blocking=True); dv.copy_(hv_, non_blocking=True)
+        din.copy_(hin, non_blocking=True)
         P.puzzle_kv_append(desc, v, dk, dv, dev_status=status, stream=stream)
         decode(desc, v, dq, sinks, out, None, num_splits=args.splits, workspace=ws,
                              dev_status=status, stream=stream)
