@@ -317,7 +317,10 @@ def run_ours(args):
                          "unit": "GB/s", "frac": round(achieved / peak, 4),
                          "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                          "us_per_launch": round(attn_mean_ms * 1e3, 2), "launches_sampled": len(attn_in_region_ms),
-                         "us_per_launch_back_to_back": round(b2b_ms * 1e3, 2), "bytes_per_launch": int(kv_bytes_attn),
+                         "us_per_launch_back_to_back": round(b2b_ms * 1e3, 2),
+                         "us_per_launch_median": round(statistics.median(attn_in_region_ms or [b2b_ms]) * 1e3, 2),
+                         "us_per_launch_min": round(min(attn_in_region_ms or [b2b_ms]) * 1e3, 2),
+                         "bytes_per_launch": int(kv_bytes_attn),
                          "read_probe_gbs": round(probe_gbs, 1),
                          "traffic": ncu_traffic(args)},
             "dev_status": dev_flags,
