@@ -34,6 +34,8 @@
 
 #include <type_traits>
 
+#include <climits>
+
 #include "common.cuh"
 #include "decode_attn.cuh"
 #include "decode_sched.cuh"
@@ -45,30 +47,30 @@ namespace {
 constexpr float kLazyLog2 = 8.0f;  // weights stay below 2^8 relative to the reference maximum
 
 
-// Producer side of one warp.  Lanes 0..NB-1 own the K block copies of a tile and lanes NB..2NB-1
-// its V block copies (NB blocks of 16 tokens per tile).  `phys` holds, per owning lane, the physical
+// Producer side of one warp.  Lane i < NB owns block i of a tile (NB blocks of 16 tokens per tile; the K copy and
+// the V copy of a block share the row coordinate).  `phys` holds, per owning lane, the physical
 // block of the NEXT tile to issue (kNotVisible: the block lies wholly outside [lo, L) and is fetched
 // from a row outside the tensor map, which the TMA unit fills with zeros).  The table entry is loaded one
 // tile ahead of its use.
 template <int TT>
 struct Producer {
   static constexpr int NB = TT / kBlock;
-  static constexpr long long kNotVisible = -(1ll << 40);  // not a value a 32-bit table entry can take
+  static constexpr int kNotVisible = INT_MIN;
   Cursor cur;
   Segment seg;
   bool ok;
-  long long phys;
+  int phys;
 
   __device__ __forceinline__ void skip_empty(const DecodeParams& P, const int* cum, const int* lens, int w) {
     while (ok && seg.t == seg.t_end) ok = next_segment<TT>(cur, seg, P, cum, lens, w);
   }
   __device__ __forceinline__ void lookup(const DecodeParams& P, int lane) {
     phys = kNotVisible;
-    if (ok && lane < 2 * NB) {
-      const int j = seg.t * NB + (lane % NB);
+    if (ok && lane < NB) {
+      const int j = seg.t * NB + lane;
       if ((j * kBlock < seg.L) && (j * kBlock + kBlock > seg.lo))
-        phys = P.block_table ? (long long)P.block_table[(size_t)seg.b * P.max_blocks_per_seq + j]
-                             : (long long)seg.b * P.max_blocks_per_seq + j;
+        phys = P.block_table ? P.block_table[(size_t)seg.b * P.max_blocks_per_seq + j]
+                             : seg.b * P.max_blocks_per_seq + j;
     }
   }
   __device__ __forceinline__ void start(Cursor c, const DecodeParams& P, const int* cum, const int* lens, int w,
@@ -84,23 +86,24 @@ struct Producer {
                                         uint32_t stage_addr, uint32_t bar) {
     if (!ok) return false;
     int row = P.oob_row;
-    if (lane < 2 * NB) {
+    if (lane < NB) {
       if (phys >= 0 && phys < P.num_blocks) {
-        row = (int)((phys * P.Hkv + seg.kvh) * P.rows_per_block);
+        row = (phys * P.Hkv + seg.kvh) * P.rows_per_block;
       } else if (phys != kNotVisible) {
         if (P.dev_status) atomicOr(P.dev_status, (int)PUZZLE_DEV_BAD_BLOCK);
       }
     }
     // the copies are issued by one lane, which collects the row coordinates first: a TMA instruction takes
     // warp-uniform operands, so issuing from several lanes would be serialised lane by lane anyway
-    int rows[2 * NB];
+    int rows[NB];
 #pragma unroll
-    for (int i = 0; i < 2 * NB; ++i) rows[i] = __shfl_sync(0xffffffffu, row, i);
+    for (int i = 0; i < NB; ++i) rows[i] = __shfl_sync(0xffffffffu, row, i);
     if (lane == 0) {
       mbar_arrive_expect_tx(bar, 2 * NB * BLOCK_BYTES);
 #pragma unroll
-      for (int i = 0; i < 2 * NB; ++i)
-        tma_load_2d(stage_addr + i * BLOCK_BYTES, i < NB ? &P.tmK : &P.tmV, 0, rows[i], bar);
+      for (int i = 0; i < NB; ++i) tma_load_2d(stage_addr + i * BLOCK_BYTES, &P.tmK, 0, rows[i], bar);
+#pragma unroll
+      for (int i = 0; i < NB; ++i) tma_load_2d(stage_addr + (NB + i) * BLOCK_BYTES, &P.tmV, 0, rows[i], bar);
     }
     if (++seg.t == seg.t_end) {
       ok = next_segment<TT>(cur, seg, P, cum, lens, w);
