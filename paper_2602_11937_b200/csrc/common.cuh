@@ -57,6 +57,17 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
   return false;
 }
 
+// True in exactly one lane of a converged warp (all 32 lanes must call it).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // ------------------------------------------------------------- TMA (tiled) --
 // 2-D tiled load global -> shared, completion counted in bytes on an mbarrier.
 // crd0 (innermost, bytes for u8 maps) must keep crd0 * element size a multiple of 16.

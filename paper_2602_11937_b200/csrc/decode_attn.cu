@@ -98,7 +98,7 @@ struct Producer {
     int rows[NB];
 #pragma unroll
     for (int i = 0; i < NB; ++i) rows[i] = __shfl_sync(0xffffffffu, row, i);
-    if (lane == 0) {
+    if (elect_one()) {
       mbar_arrive_expect_tx(bar, 2 * NB * BLOCK_BYTES);
 #pragma unroll
       for (int i = 0; i < NB; ++i) tma_load_2d(stage_addr + i * BLOCK_BYTES, &P.tmK, 0, rows[i], bar);
