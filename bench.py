@@ -365,8 +365,8 @@ def cpu_baseline(w, layer, seq_lens_host, q, sinks, window, pairs: int = 128):
 NCU_CAPTURE = {
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn.cu", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "873e8bdb34f774246fe23020f541aa43a28396e833d6749ec2ac0a2eacc17402",
-    "dram_bytes_per_launch": 1075619000 + 4381952,
+    "sha256": "5203d81a2029153ec351683a5ac8f31021eecfe3dfcd1ce272e97abaa1d321d1",
+    "dram_bytes_per_launch": 1075472000 + 4413440,
 }
 
 
