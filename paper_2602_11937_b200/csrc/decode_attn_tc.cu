@@ -259,7 +259,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
     const uint32_t my_bytes = (uint32_t)((2 * NBLK - cw + CW - 1) / CW) * 1024u;
     int n = 0;
     bool dead = false;
-    while (!dead && !C->abort && next_segment<TT>(cur, seg, P, cum, lens, w)) {
+    while (!dead && next_segment<TT>(cur, seg, P, cum, lens, w)) {   // aborts are seen warp-wide below
       if (seg.t == seg.t_end) continue;
       int row_next = lookup(seg, seg.t);
       for (int t0 = seg.t; t0 < seg.t_end && !dead; t0 += 4) {
@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
         const int nt = min(4, seg.t_end - t0);
         for (int i = 0; i < nt; ++i, ++n) {
           const int s = n % S;
-          if (C->abort || !mbar_wait_bounded(smem_u32(&ctl->kv_empty[s]), ((uint32_t)(n / S) & 1u) ^ 1u)) {
+          if (!__all_sync(kFull, !C->abort && mbar_wait_bounded(smem_u32(&ctl->kv_empty[s]), ((uint32_t)(n / S) & 1u) ^ 1u))) {
             if (!C->abort) give_up();
             dead = true;
             break;
@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
           int rows[kMine];
 #pragma unroll
           for (int k = 0; k < kMine; ++k) rows[k] = __shfl_sync(kFull, row_cur, 8 * i + ((cw + CW * k) & 7));
-          if (lane == 0) {
+          if (elect_one()) {
             const uint32_t bar = smem_u32(&ctl->kv_full[s]);
             const uint32_t dst = gbase + s * STAGE;
             mbar_arrive_expect_tx(bar, my_bytes);
@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
     // tile is issued as soon as its P is in shared memory.  The first S of a run is issued only once every
     // P.V of the runs before it has been issued: the softmax warps write the run's query rows after they have
     // finished the run before, which needs those products.
-    if (lane == 0) {
+    {
       constexpr uint32_t kIdescQK = (1u << 4) | (2u << 17) | (8u << 24);   // f32; both K-major; N = 16, M = 128
       constexpr uint32_t kIdescPV = (1u << 4) | (1u << 15) | (1u << 16) | (4u << 17) | (4u << 24);  // MN-major; N = 32, M = 64
       const uint32_t td = tmem + g * kTmemCols;
@@ -311,21 +311,25 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
       int qn = 0, qt = q_on ? qseg.t : 0, qsegno = 0;   // S = K Q^T: tiles issued, next tile, runs started
       int pn = 0, pt = p_on ? pseg.t : 0;               // O^T += V^T P likewise
       bool dead = false;
-      while ((q_on || p_on) && !dead && !C->abort) {
+      while ((q_on || p_on) && !dead) {   // an abort raised elsewhere is seen by the warp-wide checks below
         while (q_on && qn < pn + 2 && (qt != qseg.t || qn == pn)) {
           const int s = qn % S, b = qn & 1;
           bool ok = true;
           if (qt == qseg.t) ok = mbar_wait_bounded(smem_u32(&ctl->q_full), (uint32_t)qsegno & 1u);
           ok = ok && mbar_wait_bounded(smem_u32(&ctl->kv_full[s]), (uint32_t)(qn / S) & 1u) &&
                mbar_wait_bounded(smem_u32(&ctl->d1_empty[b]), ((uint32_t)(qn >> 1) & 1u) ^ 1u);
-          if (!ok || C->abort) { if (!C->abort) give_up(); dead = true; break; }
+          ok = __all_sync(kFull, ok && !C->abort);   // one decision for the warp: the issue below is warp-collective
+          if (!ok) { if (!C->abort) give_up(); dead = true; break; }
           tc_fence_after();
           const uint32_t kaddr = gbase + s * STAGE;
+          if (elect_one()) {
 #pragma unroll
-          for (int ks = 0; ks < 2; ++ks)   // 32 dims per MMA
-            umma_e4m3(td + kS + 32 * b + 16 * ks, smem_desc(kaddr + ks * 32, 16, 512, 4),
-                      smem_desc(qbase + ks * 32, 16, 512, 4), kIdescQK, 0u);
-          umma_commit(smem_u32(&ctl->d1_full[b]));
+            for (int ks = 0; ks < 2; ++ks)   // 32 dims per MMA
+              umma_e4m3(td + kS + 32 * b + 16 * ks, smem_desc(kaddr + ks * 32, 16, 512, 4),
+                        smem_desc(qbase + ks * 32, 16, 512, 4), kIdescQK, 0u);
+            umma_commit(smem_u32(&ctl->d1_full[b]));
+          }
+          __syncwarp();
           ++qn;
           if (++qt == qseg.t_end) {
             ++qsegno;
@@ -336,18 +340,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
         if (dead || !p_on) continue;
         {
           const int s = pn % S, b = pn & 1;
-          if (!mbar_wait_bounded(smem_u32(&ctl->p_full[b]), (uint32_t)(pn >> 1) & 1u) || C->abort) {
+          if (!__all_sync(kFull, mbar_wait_bounded(smem_u32(&ctl->p_full[b]), (uint32_t)(pn >> 1) & 1u) && !C->abort)) {
             if (!C->abort) give_up();
             break;
           }
           tc_fence_after();
           const uint32_t vaddr = gbase + s * STAGE + KV_TILE, paddr = pbase + b * P_BYTES;
+          if (elect_one()) {
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)   // 32 tokens per MMA
-            umma_e4m3(td + kO + 32 * ks, smem_desc(vaddr + ks * 2048, 16, 512, 4),
-                      smem_desc(paddr + ks * 1024, 256, 128, 0), kIdescPV, pt == pseg.t ? 0u : 1u);
-          umma_commit(smem_u32(&ctl->pv_done[b]));
-          umma_commit(smem_u32(&ctl->kv_empty[s]));   // the stage: its K was consumed before this P existed
+            for (int ks = 0; ks < 4; ++ks)   // 32 tokens per MMA
+              umma_e4m3(td + kO + 32 * ks, smem_desc(vaddr + ks * 2048, 16, 512, 4),
+                        smem_desc(paddr + ks * 1024, 256, 128, 0), kIdescPV, pt == pseg.t ? 0u : 1u);
+            umma_commit(smem_u32(&ctl->pv_done[b]));
+            umma_commit(smem_u32(&ctl->kv_empty[s]));   // the stage: its K was consumed before this P existed
+          }
+          __syncwarp();
           ++pn;
           if (++pt == pseg.t_end) {
             p_on = next_run(pcur, pseg);
