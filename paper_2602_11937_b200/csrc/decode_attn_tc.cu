@@ -53,12 +53,8 @@ constexpr int CW = 1;                      // copy warps per worker (1 or 3: box
 constexpr int HW = CW + 1;                 // helper warps per worker: the copy warps and one that issues the MMAs
 constexpr int kThreads = (HW * G + SW * G) * 32;
 static_assert((HW * G) % 4 == 0, "softmax warp i must have i % 4 = its tensor-memory lane quadrant");
-// Tensor memory of a worker (columns): S = K Q^T as two buffers x two 32-dim slices x 16 columns, then O^T as four
-// 32-token slices x 32 columns.  Every slice of a product has an accumulator of its own (no MMA depends on
-// another one's result); the slices are added when they are read.
-constexpr int kSlices = TT / 32;
-constexpr int kS = 0, kO = 64, kTmemCols = 256;
-static_assert(kO + 32 * kSlices <= kTmemCols, "tensor-memory layout");
+// Tensor memory of a worker (columns): S = K Q^T as two buffers of 16 columns, then O^T as 32 columns.
+constexpr int kS = 0, kO = 32, kTmemCols = 64;
 constexpr float kLazyLog2 = 8.0f;
 constexpr unsigned kFull = 0xffffffffu;
 static_assert(GROUP_BYTES % 1024 == 0, "stage bases must keep the swizzle alignment");
@@ -197,8 +193,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
     tma_prefetch_desc(&P.tmK);
     tma_prefetch_desc(&P.tmV);
   }
-  if (warp == 0) {  // owns the tensor-memory allocation: 256 columns per worker
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&C->tmem_base))
+  if (warp == 0) {  // owns the tensor-memory allocation: 64 columns per worker
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 128;" ::"r"(smem_u32(&C->tmem_base))
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -325,8 +321,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
           if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks)   // 32 dims per MMA
-              umma_e4m3(td + kS + 32 * b + 16 * ks, smem_desc(kaddr + ks * 32, 16, 512, 4),
-                        smem_desc(qbase + ks * 32, 16, 512, 4), kIdescQK, 0u);
+              umma_e4m3(td + kS + 16 * b, smem_desc(kaddr + ks * 32, 16, 512, 4),
+                        smem_desc(qbase + ks * 32, 16, 512, 4), kIdescQK, (uint32_t)ks);
             umma_commit(smem_u32(&ctl->d1_full[b]));
           }
           __syncwarp();
@@ -349,8 +345,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
           if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)   // 32 tokens per MMA
-              umma_e4m3(td + kO + 32 * ks, smem_desc(vaddr + ks * 2048, 16, 512, 4),
-                        smem_desc(paddr + ks * 1024, 256, 128, 0), kIdescPV, pt == pseg.t ? 0u : 1u);
+              umma_e4m3(td + kO, smem_desc(vaddr + ks * 2048, 16, 512, 4),
+                        smem_desc(paddr + ks * 1024, 256, 128, 0), kIdescPV, (pt == pseg.t && ks == 0) ? 0u : 1u);
             umma_commit(smem_u32(&ctl->pv_done[b]));
             umma_commit(smem_u32(&ctl->kv_empty[s]));   // the stage: its K was consumed before this P existed
           }
@@ -439,25 +435,27 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
         const int b = n & 1;
         if (!d1_ready && !mbar_wait_bounded(smem_u32(&ctl->d1_full[b]), (uint32_t)(n >> 1) & 1u)) { give_up(); dead = true; break; }
         tc_fence_after();
-        uint32_t r[8], r1[8];   // the two 32-dim slices of the dot products
-        tmem_ld8(td + kS + 32 * b + 8 * hh, r);
-        tmem_ld8(td + kS + 32 * b + 16 + 8 * hh, r1);
+        uint32_t r[8];
+        tmem_ld8(td + kS + 16 * b + 8 * hh, r);
         tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 8; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r1[i]));
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctl->d1_empty[b]));
         // ---- logits (log2 units); does the reference maximum still cover this warp's rows?
         const int tok = t * TT + row;
-        const bool visible = tok >= seg.lo && tok < seg.L;
         float tl[4];
         bool fits = true;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float raw_l = fmaf(__uint_as_float(r[4 + i]), a_lo[i], __uint_as_float(r[i]) * a_hi[i]);
-          tl[i] = visible ? raw_l : -INFINITY;     // codes of keys outside [lo, L) may be anything
+          tl[i] = fmaf(__uint_as_float(r[4 + i]), a_lo[i], __uint_as_float(r[i]) * a_hi[i]);
           fits = fits && (tl[i] <= m_ref[i] + kLazyLog2);
+        }
+        if (t * TT < seg.lo || t * TT + TT > seg.L) {   // an edge tile: codes of keys outside [lo, L) may be anything
+          if (tok < seg.lo || tok >= seg.L) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) tl[i] = -INFINITY;
+            fits = true;
+          }
         }
         // post this warp's verdict; the group's verdict is read only after the weights have been computed, so
         // nobody waits for a slower warp while it still has work of its own
@@ -523,7 +521,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
             if (!mbar_wait_bounded(smem_u32(&ctl->pv_done[(n - 1) & 1]), (uint32_t)((n - 1) >> 1) & 1u)) { give_up(); dead = true; break; }
             tc_fence_after();
 #pragma unroll
-            for (int c2 = 0; c2 < 2 * kSlices; ++c2) {   // (token slice, 16-column half)
+            for (int c2 = 0; c2 < 2; ++c2) {   // the two 16-column halves (terms 1, 2 and terms 3, 4)
               uint32_t o[8];
               tmem_ld8(td + kO + 16 * c2 + 8 * hh, o);
               tmem_wait_ld();
@@ -574,22 +572,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
       }
       group_sync(g);
       {
-        uint32_t o0[8], o1[8];   // terms 1, 2 and terms 3, 4 of this half's heads, summed over the token slices
+        uint32_t o0[8], o1[8];   // terms 1, 2 and terms 3, 4 of this half's heads
         tmem_ld8(td + kO + 8 * hh, o0);
         tmem_ld8(td + kO + 16 + 8 * hh, o1);
         tmem_wait_ld();
-#pragma unroll
-        for (int sl = 1; sl < kSlices; ++sl) {
-          uint32_t a0[8], a1[8];
-          tmem_ld8(td + kO + 32 * sl + 8 * hh, a0);
-          tmem_ld8(td + kO + 32 * sl + 16 + 8 * hh, a1);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            o0[i] = __float_as_uint(__uint_as_float(o0[i]) + __uint_as_float(a0[i]));
-            o1[i] = __float_as_uint(__uint_as_float(o1[i]) + __uint_as_float(a1[i]));
-          }
-        }
         tc_fence_before();
         const float vs = P.v_scale ? P.v_scale[seg.kvh] : 1.f;
         if (lane < 16) {   // this quadrant's 16 rows of O^T are dims 16*wq .. 16*wq + 15
@@ -623,7 +609,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 128;" ::"r"(tmem) : "memory");
   }
 }
 
