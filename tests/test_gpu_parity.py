@@ -257,8 +257,10 @@ def test_split_partials_are_what_the_oracle_computes_per_split():
     P.puzzle_decode_attn(d, dev.view(), dev.q, None, out, None, num_splits=2, workspace=ws.view(torch.uint8))
     torch.cuda.synchronize()
     rows = 64 * 2
-    part = ws[256 // 4:]                       # the partials follow the 256-byte counter block
-    assert not ws[: 256 // 4].any()            # which a finished call leaves at zero
+    head = nbytes - rows * 65 * 4              # the partials follow the block of counters (a multiple of 256 bytes)
+    assert head > 0 and head % 256 == 0
+    part = ws[head // 4:]
+    assert not ws[:1].any()                    # the pair's arrival counter: a finished call leaves it at zero
     po = part[: rows * 64].reshape(64, 2, 64).cpu().numpy().astype(np.float64)
     pl = part[rows * 64: rows * 65].reshape(64, 2).cpu().numpy().astype(np.float64)
     for s, (t0, t1) in enumerate([(0, 128), (128, 256)]):
