@@ -42,6 +42,21 @@
 
 namespace puzzle {
 
+#ifdef PUZZLE_TIMELINE
+// Diagnostic build only (timeline.py): per warp of the FP8 kernel, nanosecond stamps of the kernel entry, the first
+// tile's arrival and the end of the tile loop, and the SM it ran on; read back with puzzle_debug_timeline.
+constexpr int kTimelineWarps = 4096;
+__device__ unsigned long long g_timeline[kTimelineWarps][4];
+__device__ __forceinline__ unsigned long long timeline_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define TIMELINE(x) x
+#else
+#define TIMELINE(x)
+#endif
+
 namespace {
 
 constexpr float kLazyLog2 = 8.0f;  // weights stay below 2^8 relative to the reference maximum
@@ -167,6 +182,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
   constexpr int PIPE_BYTES = NW * NS * STAGE_BYTES;
   constexpr int NT = TT / 8;                            // 8-token n-tiles of S^T per tile
 
+  TIMELINE(const unsigned long long tl_start = timeline_now(); unsigned long long tl_first = 0;)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);
@@ -328,6 +344,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
         failed = true;
         break;
       }
+      TIMELINE(if (tl_first == 0) tl_first = timeline_now();)
       --inflight;
       const uint32_t kbase = pipe + stage * STAGE_BYTES;
       const uint32_t vbase = kbase + NB * BLOCK_BYTES;
@@ -499,6 +516,11 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     arrive_and_merge(P, cs.b, cs.kvh, cum, nW, lane);
   }
 
+  TIMELINE(if (FP8 && lane == 0 && w < kTimelineWarps) {
+    unsigned smid;
+    asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+    g_timeline[w][0] = tl_start; g_timeline[w][1] = tl_first; g_timeline[w][2] = timeline_now(); g_timeline[w][3] = smid;
+  })
   // sequences without any visible key have no tile and hence no worker in the balanced schedule
   if (!failed && P.num_splits == 0) {
     for (int p = w; p < P.batch * P.Hkv; p += nW) {
@@ -545,3 +567,10 @@ cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaSt
 }
 
 }  // namespace puzzle
+
+#ifdef PUZZLE_TIMELINE
+// Copies the stamps of the last FP8 launch to the host: unsigned long long [4096][4] (diagnostic build only).
+extern "C" __attribute__((visibility("default"))) int puzzle_debug_timeline(unsigned long long* host_out) {
+  return (int)cudaMemcpyFromSymbol(host_out, puzzle::g_timeline, sizeof(puzzle::g_timeline));
+}
+#endif
