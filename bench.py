@@ -365,7 +365,7 @@ def cpu_baseline(w, layer, seq_lens_host, q, sinks, window, pairs: int = 128):
 NCU_CAPTURE = {
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn.cu", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "5203d81a2029153ec351683a5ac8f31021eecfe3dfcd1ce272e97abaa1d321d1",
+    "sha256": "b761b1d7f16384a72e8e4be46a8eb5f45977dbdbd6f9aa513875ae08bfdf039e",
     "dram_bytes_per_launch": 1075472000 + 4413440,
 }
 
