@@ -60,16 +60,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
-TIMELINE_LIB = os.path.join(LIB_DIR, "libpuzzle_attn_timeline.so")
-
-
-def build_timeline() -> str:
-    """The same sources with -DPUZZLE_TIMELINE (per-warp time stamps in the default split-KV kernel), as a
-    separate library for timeline.py; the product library is not touched."""
-    os.makedirs(LIB_DIR, exist_ok=True)
-    subprocess.check_call([NVCC, *FLAGS, "-DPUZZLE_TIMELINE", "-shared", "-o", TIMELINE_LIB, *sources()])
-    return TIMELINE_LIB
-
-
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

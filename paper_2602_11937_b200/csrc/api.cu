@@ -31,7 +31,8 @@ EncodeTiledFn encode_tiled() {
 
 struct DeviceInfo {
   int sm_count = 0;
-  int smem_limit[3] = {0, 0, 0};  // per split-KV kernel (FP8 mma.sync, bf16, FP8 tensor-memory); 0 = not raised yet
+  // per split-KV kernel (warp-scheduled FP8, bf16; tensor-memory FP8; CTA-balanced FP8, bf16); 0 = not raised yet
+  int smem_limit[5] = {0, 0, 0, 0, 0};
 };
 DeviceInfo& device_info() {
   static DeviceInfo info[64];
@@ -95,13 +96,24 @@ int grid_ctas() { return device_info().sm_count > 0 ? device_info().sm_count : 1
 
 int decode_warps(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kDecodeWarpsFp8 : kDecodeWarpsBf16; }
 
-// The workspace starts with one arrival counter per (sequence, KV head), padded to 256 bytes.
-size_t counter_bytes(int batch, int Hkv) { return (((size_t)batch * Hkv * sizeof(int32_t)) + 255) & ~(size_t)255; }
+// The workspace starts with one arrival counter per (sequence, KV head) and the CTA-speed words of the CTA-balanced
+// kernel, padded to 256 bytes.
+size_t counter_bytes(int batch, int Hkv) {
+  return (((size_t)batch * Hkv + cta_rate_words(grid_ctas())) * sizeof(int32_t) + 255) & ~(size_t)255;
+}
+
+// The balanced schedule runs on the CTA-balanced kernel when the batch fits its shared-memory schedule.
+bool use_cta_kernel(int batch, int num_splits) { return num_splits == 0 && batch <= kCtaMaxBatch; }
 
 size_t workspace_floats(int batch, int Hkv, int num_splits, int kv_dtype) {
-  const size_t rows = num_splits == 0
-                          ? ((size_t)grid_ctas() * decode_warps(kv_dtype) + (size_t)batch * Hkv) * kGroup
-                          : (size_t)batch * Hkv * kGroup * num_splits;
+  size_t rows;
+  if (num_splits == 0) {
+    // one row block per (worker, pair) meeting of the warp-scheduled kernels (the CTA-balanced kernel needs one
+    // per (CTA, pair) meeting only, the tensor-memory kernel one per (worker, pair) with fewer workers)
+    rows = ((size_t)grid_ctas() * decode_warps(kv_dtype) + (size_t)batch * Hkv) * kGroup;
+  } else {
+    rows = (size_t)batch * Hkv * kGroup * num_splits;
+  }
   return rows * (kHeadDim + 1);
 }
 
@@ -228,8 +240,14 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   P.rows_per_block = rows_per_block;
   P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
 
-  const cudaError_t le = tc ? launch_decode_attn_tc(P, ctas, s, device_info().smem_limit + 2)
-                            : launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
+  cudaError_t le;
+  if (tc) {
+    le = launch_decode_attn_tc(P, ctas, s, device_info().smem_limit + 2);
+  } else if (use_cta_kernel(batch, num_splits)) {
+    le = launch_decode_attn_cta(P, fp8, ctas, s, device_info().smem_limit + 3);
+  } else {
+    le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
+  }
   if (le != cudaSuccess) return PUZZLE_ERR_CUDA;
   count_launch();
 

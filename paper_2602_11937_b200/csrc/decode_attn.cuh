@@ -45,17 +45,22 @@ struct MergeParams {
 
 // Shape of the two split-KV kernel variants: warps per CTA (each an independent worker), TMA stages per
 // warp and tokens per tile (the unit of the schedule and of one pipeline stage).
-#ifndef PUZZLE_FP8_WARPS
-#define PUZZLE_FP8_WARPS 12
-#define PUZZLE_FP8_STAGES 2
-#define PUZZLE_FP8_TILE 64
-#endif
-constexpr int kDecodeWarpsFp8 = PUZZLE_FP8_WARPS, kDecodeStagesFp8 = PUZZLE_FP8_STAGES, kTileFp8 = PUZZLE_FP8_TILE;
+constexpr int kDecodeWarpsFp8 = 12, kDecodeStagesFp8 = 2, kTileFp8 = 64;
 constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
+// The CTA-balanced kernel keeps its schedule arrays beside the TMA rings and the deposit buffers in shared memory,
+// which bounds the batch it takes.  Launches with at least kCtaRateMinTiles tiles per CTA note the speed of every
+// CTA slot in the workspace (after the arrival counters: a CTA counter, the buffer switch, two pad words, then two
+// float buffers of one speed per CTA) and are cut by the speeds the launch before them noted.
+constexpr int kCtaMaxBatch = 1024;
+constexpr int kCtaRateMinTiles = 256;
+inline size_t cta_rate_words(int ctas) { return 4 + 2 * (size_t)ctas; }
 
 // Launches the split-KV kernel for an FP8 (fp8 = true) or bf16 cache on `ctas` CTAs.  smem_limit[2] caches,
 // per variant, the dynamic shared-memory limit set for the kernel on the current device (0 = not set yet).
 cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit);
+// The CTA-balanced kernel (balanced schedule only, batch <= kCtaMaxBatch).  Its partial row blocks: one per
+// (CTA, pair) meeting, ctas + batch*Hkv at most.
+cudaError_t launch_decode_attn_cta(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit);
 // The tensor-memory (tcgen05) kernel for the FP8 cache.  Its tensor maps view the cache as rows of 64 bytes
 // (one token), box = 16 rows, 64-byte swizzle; P.rows_per_block is 16 and P.oob_row counts such rows.
 cudaError_t launch_decode_attn_tc(const DecodeParams& P, int ctas, cudaStream_t s, int* smem_limit);

@@ -600,7 +600,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
     if (!dead && !C->abort && P.num_splits == 0 && gi < 32) {
       for (int p = w; p < P.batch * Hkv; p += nW) {
         const int b = p / Hkv;
-        if (cum[b + 1] == cum[b]) merge_rows(P, b, p - b * Hkv, 0, 0, 0, 0, lane);
+        if (cum[b + 1] == cum[b]) merge_rows(P, b, p - b * Hkv, 0, 0, 0, 0, 0, 0, 0, lane);
       }
     }
   }

@@ -10,12 +10,6 @@
 namespace puzzle {
 namespace {
 
-__device__ __forceinline__ uint32_t f32x2_to_bf16x2(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-
 struct Segment {
   int b, kvh;
   int t, t_end;       // tiles [t, t_end) of sequence b (absolute tile index)
@@ -74,17 +68,21 @@ __device__ __forceinline__ bool next_segment(Cursor& cur, Segment& s, const Deco
 // Log-sum-exp merge of the `count` partials of one (sequence, KV head) by one warp: the quad of lanes with
 // g = lane/4 owns query head g of the group, lane c = lane%4 of the quad owns channels 16c..16c+15.
 //   M = max(sink, max_k lse_k);  Z = e^(sink-M) + sum_k e^(lse_k-M);  out = sum_k e^(lse_k-M) o_k / Z.
-// Part k of head g is partial row first + g*hstride + k*kstride.  The partials were written by other SMs
-// in this launch, so they are read past L1.
+// Part k < count of head g is partial row first + g*hstride + k*kstride; parts count .. count+count2-1 form a
+// second run, first2 + g*hstride + (k-count)*kstride2.  The partials were written by other SMs in this launch,
+// so they are read past L1.
 __device__ __noinline__ void merge_rows(const DecodeParams& P, int b, int kvh, long long first, int count,
-                                           int kstride, int hstride, int lane) {
+                                        int kstride, int hstride, long long first2, int count2, int kstride2,
+                                        int lane) {
   const int g = lane >> 2, c = lane & 3;
   const int Hq = P.Hkv * kGroup, head = kvh * kGroup + g;
   const long long row_out = (long long)b * Hq + head;
   const float sink = P.sinks ? P.sinks[head] : -INFINITY;
-  const long long base = first + (long long)g * hstride;
+  const long long base = first + (long long)g * hstride, base2 = first2 + (long long)g * hstride;
+  const int total = count + count2;
+  auto row_of = [&](int k) { return k < count ? base + (long long)k * kstride : base2 + (long long)(k - count) * kstride2; };
   float M = -INFINITY;
-  for (int k = c; k < count; k += 4) M = fmaxf(M, __ldcg(P.part_lse + base + (long long)k * kstride));
+  for (int k = c; k < total; k += 4) M = fmaxf(M, __ldcg(P.part_lse + row_of(k)));
   M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
   M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
   M = fmaxf(M, sink);
@@ -95,13 +93,13 @@ __device__ __noinline__ void merge_rows(const DecodeParams& P, int b, int kvh, l
   if (M != -INFINITY) {
     // four parts per round, every load of the round issued before the first use: the merge is a chain of
     // L2 round trips, so their number, not the arithmetic, sets its duration
-    for (int k0 = 0; k0 < count; k0 += 4) {
+    for (int k0 = 0; k0 < total; k0 += 4) {
       float l[4];
       float4 v[4][4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const bool on = k0 + j < count;
-        const long long idx = base + (long long)(on ? k0 + j : k0) * kstride;
+        const bool on = k0 + j < total;
+        const long long idx = row_of(on ? k0 + j : k0);
         l[j] = on ? __ldcg(P.part_lse + idx) : -INFINITY;
         const float4* o = reinterpret_cast<const float4*>(P.part_o + idx * kHeadDim + 16 * c);
 #pragma unroll
@@ -168,7 +166,7 @@ __device__ __forceinline__ void arrive_and_merge(const DecodeParams& P, int b, i
   last = __shfl_sync(0xffffffffu, last, 0);
   if (!last) return;
   __threadfence();  // the arrivals before the other warps' partials are read
-  merge_rows(P, b, kvh, first, count, kstride, hstride, lane);
+  merge_rows(P, b, kvh, first, count, kstride, hstride, 0, 0, 0, lane);
   if (lane == 0) P.counters[p] = 0;
 }
 

@@ -13,6 +13,7 @@ import torch
 import oracle
 import synth
 from helpers import bf16_bits
+from gpu_helpers import assert_close
 
 pytestmark = pytest.mark.gpu
 
@@ -116,7 +117,9 @@ def test_full_size_128k_context(kv_dtype):
 
 
 def test_stack_driver_matches_layer_by_layer_calls():
-    """The per-layer pattern driver (eager and as a CUDA graph) gives what the single calls give."""
+    """The per-layer pattern driver (eager and as a CUDA graph) gives what the single calls give.  Tiles are handed
+    to warps as they become free, so the order of the float32 sums, and with it the last bit of a bf16 output, may
+    differ between two runs on the same inputs: the comparison uses the parity bound, not bit equality."""
     import paper_2602_11937_b200 as P
     from synth.device import fill_layer
     w = synth.workload(4, scale=0.03)                     # batch 2, ragged contexts up to 1475
@@ -140,14 +143,16 @@ def test_stack_driver_matches_layer_by_layer_calls():
     out = [torch.zeros_like(r) for r in ref]
     stack.step(q, [a for a, _ in kv], [b for _, b in kv], out)
     torch.cuda.synchronize()
-    for o, r in zip(out, ref):
-        assert torch.equal(o, r)
+    for i, (o, r) in enumerate(zip(out, ref)):
+        assert_close(o.float().cpu().numpy().astype(np.float64), r.float().cpu().numpy().astype(np.float64),
+                     "eager stack, layer %d" % i)
     out2 = [torch.zeros_like(r) for r in ref]
     g = stack.capture(q, [a for a, _ in kv], [b for _, b in kv], out2)
     for o in out2:
         o.zero_()
     g.replay()
     torch.cuda.synchronize()
-    for o, r in zip(out2, ref):
-        assert torch.equal(o, r)
+    for i, (o, r) in enumerate(zip(out2, ref)):
+        assert_close(o.float().cpu().numpy().astype(np.float64), r.float().cpu().numpy().astype(np.float64),
+                     "captured stack, layer %d" % i)
     assert int(stack.status.item()) == 0

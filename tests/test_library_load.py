@@ -36,7 +36,9 @@ def test_status_strings_and_workspace_size_need_no_gpu():
     d = P.layer_desc()
     a = P.puzzle_decode_attn_workspace_bytes(d, 16, 0)
     b = P.puzzle_decode_attn_workspace_bytes(d, 16, 8)
-    assert a > 0 and b == 512 + 16 * 64 * 8 * 65 * 4   # counters (16*8 int32, padded to 256) + partials
+    partials = 16 * 64 * 8 * 65 * 4                     # 8 splits of (o, lse) per (sequence, query head)
+    head = b - partials                                 # arrival counters + CTA-speed words (these grow with the SM count)
+    assert a > 0 and head % 256 == 0 and head >= (16 * 8 + 4 + 2) * 4
     bad = P.layer_desc(head_dim=128)
     assert P.puzzle_decode_attn_workspace_bytes(bad, 16, 0) == 0
 
