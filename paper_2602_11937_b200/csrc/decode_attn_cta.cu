@@ -279,6 +279,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
   CtaCtl& ctl = *reinterpret_cast<CtaCtl*>(sp);                           sp += sizeof(CtaCtl);
   const uint32_t ctl_a = smem_u32(&ctl);
   int* bound = reinterpret_cast<int*>(sp);                                sp += ((nC + 1 + 3) & ~3) * sizeof(int);
+  int* share = reinterpret_cast<int*>(sp);                                sp += ((nC + 1 + 3) & ~3) * sizeof(int);
   int* cum = reinterpret_cast<int*>(sp);
 
   // speeds of the CTA slots from earlier launches: two buffers, the valid one named by `epoch`
@@ -306,8 +307,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
   if (threadIdx.x < 32) dep_piece[threadIdx.x] = -1;
   if (threadIdx.x < kPieceSlots) { pk_key[threadIdx.x] = -1; pk_done[threadIdx.x] = 0; }
   if (threadIdx.x == 0) cum[0] = 0;
-  // one warp turns the noted speeds into cumulative shares (fixed point, 4096 = the mean speed), kept in bound[]
-  // until the tile count is known; without a full set of speeds every CTA gets the same share
+  // one warp turns the noted speeds into cumulative shares (fixed point, 4096 = the mean speed); without a full set
+  // of speeds every CTA gets the same share
   if (warp == 1) {
     const int ep = *reinterpret_cast<const volatile int*>(epoch_p) & 1;
     float r[8];
@@ -337,10 +338,10 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
         const int u = __shfl_up_sync(0xffffffffu, v, d);
         if (lane >= d) v += u;
       }
-      if (cc < nC) bound[cc + 1] = v + carry;  // cumulative share up to and including CTA cc
+      if (cc < nC) share[cc + 1] = v + carry;  // cumulative share up to and including CTA cc
       carry += __shfl_sync(0xffffffffu, v, 31);
     }
-    if (lane == 0) bound[0] = 0;
+    if (lane == 0) share[0] = 0;
   }
   __syncthreads();
   // ---- step 2 (one warp): prefix sums
@@ -361,38 +362,35 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
   __syncthreads();
   // ---- step 3: range boundaries of all CTAs (the merge needs them), and this CTA's hand-out state.
   // Large launches are cut in proportion to the CTA speeds; small ones evenly over as many CTAs as there are tiles.
+  // Every CTA evaluates the same expressions on the same numbers, so all agree on the cuts.
   {
     const int T = cum[P.batch];
     const bool large = T / nC >= kCtaRateMinTiles && nC <= 256;
     const int nR = large ? nC : max(1, min(nC, T));
     const int snap = max(1, (T / nR) >> 5);
-    const long long share_total = bound[nC];
-    // thread i computes boundary i (and keeps it while the shares in bound[] are still being read by others)
-    for (int base = 0; base <= nC; base += blockDim.x) {
-      const int i = base + threadIdx.x;
-      int x = 0;
-      if (i <= nC) {
-        if (i == 0) x = 0;
-        else if (i >= nR) x = T;
-        else {
-          x = large ? (int)(((long long)bound[i] * T) / share_total) : (int)(((long long)i * T) / nR);
-          if (x > 0 && x < T) x = snap_cut(cum, P.batch, P.Hkv, x, snap);
-        }
-      }
-      __syncthreads();
-      if (i <= nC) bound[i] = x;
-      __syncthreads();
-    }
-    if (threadIdx.x == 32) {
-      ctl.lo = bound[blockIdx.x];
-      ctl.end = bound[blockIdx.x + 1];
-      ctl.pos = ctl.lo;
-      int pf = 0;
-      if (ctl.lo < ctl.end) {
-        const int b = seq_of(cum, P.batch, ctl.lo);
-        pf = b * P.Hkv + (ctl.lo - cum[b]) / ((cum[b + 1] - cum[b]) / P.Hkv);
+    const float per_share = (float)T / (float)share[nC];
+    auto boundary = [&](int i) {
+      if (i <= 0) return 0;
+      if (i >= nR) return T;
+      // small launches on up to 256 CTAs: i * T < 2^24 (fewer than kCtaRateMinTiles tiles per CTA)
+      const int x = large ? min(T - 1, (int)((float)share[i] * per_share))
+                          : (nC <= 256 ? (i * T) / nR : (int)(((long long)i * T) / nR));
+      return x > 0 ? snap_cut(cum, P.batch, P.Hkv, x, snap) : 0;
+    };
+    for (int i = threadIdx.x; i <= nC; i += blockDim.x) bound[i] = boundary(i);
+    // two threads of otherwise idle warps work out this CTA's own range at the same time
+    if (threadIdx.x == 32 * (NW - 1)) {
+      const int lo_c = boundary(blockIdx.x);
+      ctl.lo = ctl.pos = lo_c;
+      int pf = 0;  // the pair the range starts in (unused when the range is empty)
+      if (lo_c < T) {
+        const int b = seq_of(cum, P.batch, lo_c);
+        pf = b * P.Hkv + (lo_c - cum[b]) / ((cum[b + 1] - cum[b]) / P.Hkv);
       }
       ctl.p_first = pf;
+    }
+    if (threadIdx.x == 32 * (NW - 2)) {
+      ctl.end = boundary(blockIdx.x + 1);
       ctl.warps_left = NW;
       ctl.use_rates = large ? 1 : 0;
     }
@@ -639,7 +637,7 @@ static size_t cta_smem_bytes(int batch, int ctas) {
   return 1024 + (size_t)NW * NS * STAGE_BYTES + NW * NS * 8 + (size_t)NW * NS * sizeof(TileDesc) +
          NW * sizeof(TileDesc) + NW * sizeof(PairCache) + (size_t)NW * 4 * 32 * sizeof(float4) +
          2 * NW * kGroup * sizeof(float) + 32 * sizeof(int) + 2 * kPieceSlots * sizeof(int) + sizeof(CtaCtl) +
-         (size_t)((ctas + 1 + 3) & ~3) * sizeof(int) + (size_t)(batch + 1) * sizeof(int);
+         2 * (size_t)((ctas + 1 + 3) & ~3) * sizeof(int) + (size_t)(batch + 1) * sizeof(int);
 }
 
 template <int NW, int NS, int TT, bool FP8>
