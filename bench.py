@@ -130,6 +130,37 @@ def shard_workload(w: synth.Workload, rank: int, world: int) -> synth.Workload:
     return w
 
 
+def shard_plan(w: synth.Workload, seq_lens, rank: int, world: int, mode: str):
+    """What rank `rank` of `world` holds and moves in one layer-step under the three ways the path shards
+    (batch: its own sequences; heads: Hkv/world KV heads of every sequence; context: every world-th cache block
+    of every sequence).  Returns (workload of the rank's shard, its seq_lens for attention, its seq_lens for the
+    append, algorithmic bytes the rank moves per step).  Host arithmetic only."""
+    import dataclasses
+    from paper_2602_11937_b200.parallel import context_slice, head_slice
+    lens = torch.as_tensor(seq_lens, dtype=torch.int32)
+    window = w.windows[0]
+    if mode == "batch":
+        ws = shard_workload(dataclasses.replace(w), rank, world)
+        return ws, lens, lens, algorithmic_bytes(ws, lens.tolist(), window)
+    if mode == "heads":
+        kv, qh = head_slice(rank, world, w.hkv, w.hq // w.hkv)
+        ws = dataclasses.replace(w, hkv=kv.stop - kv.start, hq=qh.stop - qh.start)
+        return ws, lens, lens, algorithmic_bytes(ws, lens.tolist(), window)
+    if mode == "context":
+        if window != 0:
+            raise ValueError("context sharding covers full-attention layers only")
+        local, app = context_slice(lens, rank, world, w.block)
+        per_rank_blocks = (w.blocks_per_seq + world - 1) // world
+        ws = dataclasses.replace(w, context=per_rank_blocks * w.block)
+        row = 2 * w.hkv * w.head_dim
+        nbytes = sum(int(L) * row + ((int(L) + w.block - 1) // w.block) * 4 for L in local.tolist())
+        nbytes += 2 * w.batch * w.hq * w.head_dim * 2                       # q in, out (every rank has both)
+        nbytes += 3 * 2 * w.hkv * w.head_dim * int((app > 0).sum())         # new K/V read + cache write, owner only
+        nbytes += (world + 1) * w.batch * w.hq * (w.head_dim + 1) * 4 if world > 1 else 0   # partials written, gathered ones read
+        return ws, local, app, nbytes
+    raise ValueError(mode)
+
+
 def max_over_ranks(values, world: int, device):
     """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the job's time)."""
     t = torch.tensor(list(values), dtype=torch.float64, device=device)
@@ -139,36 +170,83 @@ def max_over_ranks(values, world: int, device):
     return [float(x) for x in t.tolist()]
 
 
+def sum_over_ranks(value: float, world: int, device) -> float:
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t)
+    return float(t.item())
+
+
 def job_throughput_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float) -> float:
     """Whole-job value: every rank moves bytes_per_rank_step per step, the step takes the slowest rank's time."""
     return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
 
 
-def run_ours(args):
+def launch_plan(gpus: int, env) -> tuple:
+    """How this process takes part in a run on `gpus` GPUs: ("rank", rank, local_rank, world) when a launcher
+    started it (its world size must be `gpus`), ("single",) for one GPU, ("spawn", gpus) when it has to start the
+    ranks itself.  Anything else is an error: a run never reports fewer GPUs than it was asked for."""
+    if gpus < 1:
+        raise SystemExit("--gpus must be at least 1")
+    if "WORLD_SIZE" in env:
+        world = int(env["WORLD_SIZE"])
+        if world != gpus:
+            raise SystemExit("--gpus %d, but the launcher started %d ranks" % (gpus, world))
+        return ("rank", int(env.get("RANK", "0")), int(env.get("LOCAL_RANK", "0")), world)
+    return ("single",) if gpus == 1 else ("spawn", gpus)
+
+
+def spawn_ranks(gpus: int) -> int:
+    """Re-runs this command line as `gpus` ranks under torch.distributed.run on this node; returns its exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def median_region(regions):
+    """Index of the region whose time is the median of all (the lower one of the middle two)."""
+    order = sorted(range(len(regions)), key=lambda i: regions[i])
+    return order[(len(order) - 1) // 2]
+
+
+def run_ours(args, plan):
     import paper_2602_11937_b200 as P
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local_rank, world = (plan[1], plan[2], plan[3]) if plan[0] == "rank" else (0, 0, 1)
+    if torch.cuda.device_count() <= local_rank:
+        raise SystemExit("rank %d needs GPU %d, this node shows %d" % (rank, local_rank, torch.cuda.device_count()))
     torch.cuda.set_device(local_rank)
     dev = "cuda:%d" % local_rank
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    w = shard_workload(synth.workload(args.config), rank, world)
+    mode = args.shard
+    w0 = synth.workload(args.config)
+    if mode == "context" and w0.windows[0] != 0:
+        raise SystemExit("--shard context needs a workload whose first layer is full attention")
+    seq_global = synth.draw_seq_lens(shard_workload(synth.workload(args.config), rank, world) if mode == "batch" else w0)
+    w, lens_attn, lens_append, bytes_rank = shard_plan(w0, seq_global, rank, world, mode)
     window = w.windows[0]
-    seq_lens_host = synth.draw_seq_lens(w).tolist()
-    seq_lens = torch.tensor(seq_lens_host, dtype=torch.int32, device=dev)
+    seq_lens = lens_attn.to(dev)
+    seq_append = lens_append.to(dev)
     layers = [build_layer(w, l, dev) for l in range(args.layers)]
     desc = P.layer_desc(window=window, num_q_heads=w.hq, num_kv_heads=w.hkv, head_dim=w.head_dim,
                         block_size=w.block)
     if args.contiguous:
         for L in layers:
             L["table"] = None
-    views = [P.kv_view(L["k_cache"], L["v_cache"], seq_lens, block_table=L["table"],
-                       max_blocks_per_seq=w.blocks_per_seq, k_scale=L["k_scale"], v_scale=L["v_scale"])
-             for L in layers]
+
+    def view_of(L, lens):
+        return P.kv_view(L["k_cache"], L["v_cache"], lens, block_table=L["table"], max_blocks_per_seq=w.blocks_per_seq,
+                         k_scale=L["k_scale"], v_scale=L["v_scale"])
+    views = [view_of(L, seq_lens) for L in layers]
+    views_append = views if mode != "context" else [view_of(L, seq_append) for L in layers]
     q = synth.draw_q(w, 0, dev)
     k_new, v_new = synth.draw_new_kv(w, 0, dev)
     sinks = synth.draw_sinks(w, 0, dev)
@@ -178,62 +256,82 @@ def run_ours(args):
         kernel_name = "decode_attn_tc_kernel (tcgen05 split-KV pass with the merge fused in)"
         dtype_name = "e4m3 tcgen05 mma on the cache codes, f32 accumulate and softmax"
     else:
-        kernel_name = "decode_attn_kernel<fp8> (split-KV pass with the merge fused in)"
+        kernel_name = ("decode_attn_cta_kernel<fp8>" if args.splits == 0 else "decode_attn_kernel<fp8>") + \
+            " (split-KV pass with the merge fused in)"
         dtype_name = "f16 mma on e4m3 codes, f32 accumulate and softmax"
     ws = torch.empty(P.puzzle_decode_attn_workspace_bytes(desc, w.batch, args.splits), dtype=torch.uint8, device=dev)
     P.puzzle_decode_attn_workspace_init(desc, w.batch, ws)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
+    ctx = None
+    if mode == "context":
+        from paper_2602_11937_b200.parallel import ContextShardedAttention
+        ctx = ContextShardedAttention(desc, w.batch, dev, world, num_splits=args.splits)
 
-    attn_events = []   # CUDA-event pairs around the attention launch of every 8th timed step
+    def attention(i, qq):
+        if ctx is not None:    # partial over this rank's blocks -> one all-gather -> merge with the sink
+            ctx.step(views[i % len(views)], qq, sinks, out)
+        else:
+            decode(desc, views[i % len(views)], qq, sinks, out, None, num_splits=args.splits, workspace=ws,
+                   dev_status=status, stream=stream)
 
-    def step(i, sample=False):
-        v = views[i % len(views)]
-        P.puzzle_kv_append(desc, v, k_new, v_new, dev_status=status, stream=stream)
-        if sample:
+    def step(i, events=None):
+        P.puzzle_kv_append(desc, views_append[i % len(views)], k_new, v_new, dev_status=status, stream=stream)
+        if events is not None:
             ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             ea.record(stream)
-        decode(desc, v, q, sinks, out, None, num_splits=args.splits, workspace=ws,
-                             dev_status=status, stream=stream)
-        if sample:
+        attention(i, q)
+        if events is not None:
             eb.record(stream)
-            attn_events.append((ea, eb))
+            events.append((ea, eb))
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)
+    for i in range(warmup):
         step(i)
     barrier()
 
-    # ---- timed region: device-resident inputs
+    # ---- timed regions: device-resident inputs.  A region is exactly K steps between two events, with a barrier
+    # and a device synchronise on both sides; regions are repeated until min_seconds of GPU time have passed.
+    # Regions alternate between plain ones (nothing but the steps between the two events: their median gives
+    # ms_per_step and value) and sampled ones (CUDA events around every attention launch, every 8th beyond 256
+    # steps, which cost a few microseconds per step: the median sampled region gives the kernel's launch duration).
+    every = 1 if args.steps <= 256 else 8
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
     time.sleep(0.25)
-    launches0 = P.puzzle_launch_count()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    t0.record(stream)
-    for i in range(args.steps):
-        step(i, sample=(i % 8 == 7))
-    t1.record(stream)
-    barrier()
-    launches = P.puzzle_launch_count() - launches0
-    ms_total = t0.elapsed_time(t1)
-    attn_in_region_ms = [a.elapsed_time(b) for a, b in attn_events]
-    # the attention kernel alone: the same launches back to back on the same stream, no append in between
-    n_attn = min(args.steps, 400)
-    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a0.record(stream)
-    for i in range(n_attn):
-        decode(desc, views[i % len(views)], q, sinks, out, None, num_splits=args.splits, workspace=ws,
-                             dev_status=status, stream=stream)
-    a1.record(stream)
-    barrier()
-    attn_ms = [a0.elapsed_time(a1) / n_attn]
+    plain, sampled, launch_ms, launches_per_region = [], [], [], 0
+    it = warmup
+    while True:
+        want_events = len(plain) > len(sampled)
+        events = []
+        l0 = P.puzzle_launch_count()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0.record(stream)
+        for k in range(args.steps):
+            step(it + k, events if want_events and k % every == every - 1 else None)
+        t1.record(stream)
+        barrier()
+        it += args.steps
+        launches_per_region = P.puzzle_launch_count() - l0
+        ms = max_over_ranks([t0.elapsed_time(t1)], world, dev)[0]
+        if want_events:
+            sampled.append(ms)
+            launch_ms.append([a.elapsed_time(b) for a, b in events])
+        else:
+            plain.append(ms)
+        n_regions = len(plain) + len(sampled)
+        if len(sampled) >= 1 and (sum(plain) + sum(sampled) >= args.min_seconds * 1e3 or n_regions >= args.max_regions):
+            break
     clocks = sampler.stop()
+    ms_total = plain[median_region(plain)]
+    mid = median_region(sampled)
+    regions = plain + sampled
 
     # ---- end to end: the step's inputs start in pinned host memory, the result ends there
     # q, k_new and v_new of a step travel as ONE pinned host buffer and one copy (the caller's side of the API:
@@ -246,24 +344,28 @@ def run_ours(args):
     hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
 
     def step_e2e(i):
-        v = views[i % len(views)]
         din.copy_(hin, non_blocking=True)
-        P.puzzle_kv_append(desc, v, dk, dv, dev_status=status, stream=stream)
-        decode(desc, v, dq, sinks, out, None, num_splits=args.splits, workspace=ws,
-                             dev_status=status, stream=stream)
+        P.puzzle_kv_append(desc, views_append[i % len(views)], dk, dv, dev_status=status, stream=stream)
+        attention(i, dq)
         hout.copy_(out, non_blocking=True)
 
     for i in range(3):
         step_e2e(i)
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        step_e2e(i)
-        stream.synchronize()   # the caller reads the result on the host before the next step
-    e1.record(stream)
-    barrier()
-    ms_e2e = e0.elapsed_time(e1)
+    e2e_regions = []
+    while True:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            step_e2e(i)
+            stream.synchronize()   # the caller reads the result on the host before the next step
+        e1.record(stream)
+        barrier()
+        e2e_regions.append(max_over_ranks([e0.elapsed_time(e1)], world, dev)[0])
+        if sum(e2e_regions) >= 0.5 * args.min_seconds * 1e3 or len(e2e_regions) >= args.max_regions:
+            break
+    ms_e2e = e2e_regions[median_region(e2e_regions)]
 
     # ---- read-only streaming probe (one pass over 2 GiB): the bandwidth a pure scan reaches on this device
     probe_buf = torch.empty(2 << 30, dtype=torch.uint8, device=dev)
@@ -281,52 +383,64 @@ def run_ours(args):
     probe_gbs = probe_buf.numel() / (statistics.median(probe_ms) * 1e-3) / 1e9
     del probe_buf
 
-    dev_flags = int(status.item())
-    bytes_step = algorithmic_bytes(w, seq_lens_host, window)
-    kv_bytes_attn = bytes_step - 2 * w.batch * w.hkv * w.head_dim * 3   # what the attention pass itself moves
-    # roofline: mean duration of the attention launches sampled INSIDE the timed region (falls back to the
-    # back-to-back loop when the run is too short to hold a sample)
-    b2b_ms = statistics.mean(attn_ms)
-    in_region_ms = statistics.mean(attn_in_region_ms) if attn_in_region_ms else b2b_ms
-    ms_total, ms_e2e, attn_mean_ms, b2b_ms = max_over_ranks([ms_total, ms_e2e, in_region_ms, b2b_ms], world, dev)
+    dev_flags = int(status.item()) | (int(ctx.status.item()) if ctx is not None else 0)
+    # bytes of the step on this rank; the attention pass itself moves all of them but the appended token's
+    kv_bytes_attn = bytes_rank - 2 * w.batch * w.hkv * w.head_dim * 3
+    in_region = launch_ms[mid] or [ms_total / args.steps]
+    all_launches = [x for r in launch_ms for x in r] or in_region
+    attn_mean_ms = max_over_ranks([statistics.mean(in_region)], world, dev)[0]
+    bytes_job = sum_over_ranks(float(bytes_rank), world, dev)
 
     if rank == 0:
         peak, peak_kind = measured_peak()
         ms_step = ms_total / args.steps
-        value = job_throughput_gbs(bytes_step, world, ms_step)
+        value = bytes_job / (ms_step * 1e-3) / 1e9
         achieved = kv_bytes_attn / (attn_mean_ms * 1e-3) / 1e9
+        par = {"batch": "dp%d (independent sequences per GPU, no collective)" % world,
+               "heads": "tp%d over KV heads (no collective inside the path)" % world,
+               "context": "cp%d over cache blocks (one all-gather of float32 partials, then the merge)" % world}[mode]
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5),
-            "us_per_layer_step": round(ms_step * 1e3, 2), "higher_is_better": True, "scaling": "weak",
+            "warmup": warmup, "ms_per_step": round(ms_step, 5),
+            "us_per_layer_step": round(ms_step * 1e3, 2), "higher_is_better": True,
+            "scaling": "weak" if mode == "batch" else "strong",
             "vs_baseline": None, "dtype": dtype_name, "data": "synthetic",
-            "config": {"workload": w.name, "batch_per_gpu": w.batch, "context": w.context, "q_heads": w.hq,
-                       "kv_heads": w.hkv, "head_dim": w.head_dim, "block_size": w.block, "window": window, "paged": not args.contiguous,
-                       "num_splits": args.splits, "rotating_layer_caches": len(layers),
-                       "l2": "inputs larger than L2: %.0f MiB per step, %d caches rotated" % (
-                           bytes_step / 2 ** 20, len(layers)),
-                       "parallelism": "dp%d (independent sequences per GPU, no collective)" % world},
+            "config": {"workload": w0.name, "batch_per_gpu": w.batch, "context": w0.context, "q_heads": w.hq,
+                       "kv_heads": w.hkv, "head_dim": w.head_dim, "block_size": w.block, "window": window,
+                       "paged": not args.contiguous, "num_splits": args.splits, "rotating_layer_caches": len(layers),
+                       "l2": "inputs larger than L2: %.0f MiB per step and GPU, %d caches rotated" % (
+                           bytes_rank / 2 ** 20, len(layers)),
+                       "parallelism": par},
+            "timing": {"regions_plain": len(plain), "regions_with_launch_events": len(sampled),
+                       "region_reported": "median of the plain regions (ms_per_step, value); the median region with "
+                                          "events around the attention launches gives roofline.us_per_launch",
+                       "gpu_seconds_timed": round(sum(regions) / 1e3, 3),
+                       "ms_per_step_min": round(min(plain) / args.steps, 5),
+                       "ms_per_step_max": round(max(plain) / args.steps, 5),
+                       "ms_per_step_with_launch_events": round(sampled[mid] / args.steps, 5)},
             "clocks": clocks,
-            "e2e": {"value": round(world * bytes_step / (ms_e2e / args.steps * 1e-3) / 1e9, 1), "unit": "GB/s",
-                    "ms_per_step": round(ms_e2e / args.steps, 5),
+            "e2e": {"value": round(bytes_job / (ms_e2e / args.steps * 1e-3) / 1e9, 1), "unit": "GB/s",
+                    "ms_per_step": round(ms_e2e / args.steps, 5), "regions": len(e2e_regions),
                     "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in (q, k_new, v_new))),
                     "d2h_bytes_per_step": int(out.numel() * out.element_size())},
-            "gpu_launches": int(launches),
+            "gpu_launches": int(launches_per_region),
             "roofline": {"bound": "hbm", "kernel": kernel_name,
                          "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
                          "unit": "GB/s", "frac": round(achieved / peak, 4),
                          "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
-                         "us_per_launch": round(attn_mean_ms * 1e3, 2), "launches_sampled": len(attn_in_region_ms),
-                         "us_per_launch_back_to_back": round(b2b_ms * 1e3, 2),
-                         "us_per_launch_median": round(statistics.median(attn_in_region_ms or [b2b_ms]) * 1e3, 2),
-                         "us_per_launch_min": round(min(attn_in_region_ms or [b2b_ms]) * 1e3, 2),
+                         "target_75pct_of_nominal_met": bool(achieved / NOMINAL_HBM_GBS >= 0.75),
+                         "us_per_launch": round(attn_mean_ms * 1e3, 2), "launches_sampled": len(in_region),
+                         "launches_sampled_all_regions": len(all_launches),
+                         "us_per_launch_median_all_regions": round(statistics.median(all_launches) * 1e3, 2),
+                         "us_per_launch_min_all_regions": round(min(all_launches) * 1e3, 2),
+                         "sm_mhz_median": clocks.get("sm_mhz"),
                          "bytes_per_launch": int(kv_bytes_attn),
                          "read_probe_gbs": round(probe_gbs, 1),
-                         "traffic": ncu_traffic(args)},
+                         "traffic": ncu_traffic(args), "traffic_source": NCU_CAPTURE["source"]},
             "dev_status": dev_flags,
         }
-        if args.cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w, layers[0], seq_lens_host, q, sinks, window)
+        if args.cpu_baseline and mode == "batch":
+            line["cpu_baseline"] = cpu_baseline(w, layers[0], seq_lens.tolist(), q, sinks, window)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -359,12 +473,13 @@ def cpu_baseline(w, layer, seq_lens_host, q, sinks, window, pairs: int = 128):
 # ------------------------------------------------------- 36-layer stack mode ---
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the default split-KV kernel on the
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the default (CTA-balanced) split-KV kernel on the
 # headline workload, from the one-launch `ncu --set full` capture summarised under profiles/; valid only for
 # the kernel sources it was taken from, so it is tied to their hash and reported as null once they change.
 NCU_CAPTURE = {
+    "source": "profiles/decode_attn_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
-    "sources": ("decode_attn.cu", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
+    "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
     "sha256": "b761b1d7f16384a72e8e4be46a8eb5f45977dbdbd6f9aa513875ae08bfdf039e",
     "dram_bytes_per_launch": 1075472000 + 4413440,
 }
@@ -496,10 +611,16 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200, help="steps per timed region")
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--min-seconds", type=float, default=0.5,
+                    help="timed regions of --steps steps are repeated until this much GPU time has passed")
+    ap.add_argument("--max-regions", type=int, default=400)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=3, help="workload id 1..5 (3 = batch 16, context 64K)")
+    ap.add_argument("--config", type=int, default=None, help="workload id 1..5 (default 3: batch 16, context 64K; "
+                    "5 with --shard heads|context)")
+    ap.add_argument("--shard", default="batch", choices=["batch", "heads", "context"],
+                    help="how N GPUs share the layer: own sequences each (default), KV heads, or cache blocks")
     ap.add_argument("--splits", type=int, default=0, help="0 = balanced schedule, S = fixed splits per sequence")
     ap.add_argument("--layers", type=int, default=4, help="distinct layer caches rotated between steps")
     ap.add_argument("--stack", type=int, default=0, choices=[0, 4, 5],
@@ -514,12 +635,17 @@ def main():
     ap.add_argument("--ncu-traffic", type=float, default=None,
                     help="DRAM bytes per launch of the attention kernel from an ncu capture (reported as-is)")
     args = ap.parse_args()
+    if args.config is None:
+        args.config = 3 if args.shard == "batch" else 5
+    plan = launch_plan(args.gpus, os.environ)
+    if plan[0] == "spawn":
+        sys.exit(spawn_ranks(args.gpus))
     if args.stack:
         run_stack(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
-        run_ours(args)
+        run_ours(args, plan)
 
 
 if __name__ == "__main__":
