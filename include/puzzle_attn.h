@@ -18,9 +18,16 @@
  * Conventions for every entry point
  *   - All data pointers are DEVICE pointers owned by the caller, unless marked
  *     "host".  The two descriptor structs are read on the host during the call.
- *   - Nothing is allocated, freed or kept between calls.  Work is enqueued on
- *     the CUDA stream passed as `stream` (a cudaStream_t cast to void*; NULL is
- *     the default stream) and the call returns without synchronising.
+ *   - No device memory is allocated or freed by any call; what the library
+ *     keeps between calls is host-side only (per device: its SM count, the
+ *     shared-memory limit it has set on its kernels, the address of the
+ *     built-in scratch array).  Work is enqueued on the CUDA stream passed as
+ *     `stream` (a cudaStream_t cast to void*; NULL is the default stream) and
+ *     the call returns without synchronising.
+ *   - The balanced schedule hands tiles of the cache to warps as they become
+ *     free, so the order of the float32 sums can differ between two calls on the
+ *     same inputs: outputs agree to rounding (the last bit of a bf16 value may
+ *     differ), not bit for bit.  Appended cache bytes are always bit-exact.
  *   - Errors that the host can see (NULL required pointer, unsupported shape,
  *     workspace too small) return a code BEFORE anything is launched.  A CUDA
  *     launch error maps to PUZZLE_ERR_CUDA.  Errors only the device can see
@@ -132,13 +139,24 @@ PUZZLE_API puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, 
                                  const void* k_new, const void* v_new, const int32_t* new_lens, int32_t batch,
                                  int32_t n_new, int32_t* dev_status, void* stream);
 
+/* Values of num_splits below 1: the balanced schedule, with the kernel chosen by the library or pinned. */
+#define PUZZLE_SCHED_AUTO 0
+#define PUZZLE_SCHED_CTA (-1)
+#define PUZZLE_SCHED_WARP (-2)
+
 /* Bytes of scratch puzzle_decode_attn needs for this batch and split choice
- * (0 on invalid arguments).  num_splits == 0 selects the balanced schedule. */
+ * (0 on invalid arguments).  num_splits <= 0 selects the balanced schedule.
+ * The scratch serves the split-KV pass of the KV-I/O-bound decode (paper,
+ * Section "Optimized Scenarios"): float32 partial (o, lse) rows, arrival
+ * counters, and the speeds of the CTA slots noted by large launches (see
+ * puzzle_decode_attn).  The paper does not describe a split-KV pass; the
+ * partition and its merge follow the problem statement this library was built
+ * to.  The size depends on the batch and the device's SM count, not on the
+ * context length (the grid is persistent), so there is no max_seq_len argument. */
 PUZZLE_API size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits);
 
-/* Prepares a freshly allocated workspace: zero-fills the arrival counters at
- * its start (one int32 per (sequence, KV head), padded to 256 bytes) on
- * `stream`.  Call it once per workspace before its first puzzle_decode_attn;
+/* Prepares a freshly allocated workspace: zero-fills the arrival counters and
+ * the CTA-speed words at its start (padded to 256 bytes) on `stream`.  Call it once per workspace before its first puzzle_decode_attn;
  * every completed puzzle_decode_attn leaves the counters at zero again, for any
  * batch and split choice that fits the workspace.  Call it again after a step
  * whose *dev_status reported PUZZLE_DEV_WAIT_EXPIRED (that step stopped half
@@ -160,10 +178,17 @@ PUZZLE_API puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_de
  *   q: bf16 [batch][num_q_heads][head_dim], 8-byte aligned;  sinks: float32 [num_q_heads] or NULL (no sink);
  *   out: bf16 [batch][num_q_heads][head_dim], 16-byte aligned;  lse_out: float32 [batch][num_q_heads] or NULL;
  *   num_splits: 0 = balanced schedule (recommended); S >= 1 = every (sequence, KV head) context is
- *     cut into S equal runs of 64-token tiles;
+ *     cut into S equal runs of 64-token tiles.  The balanced schedule has two kernels and picks by
+ *     what the host knows about the size of the launch (batch, window, block-table row length):
+ *     large launches are cut into one range of tiles per CTA, handed out to its warps as they become
+ *     free, in proportion to the speed each CTA showed in the previous large launch on this
+ *     workspace; small ones (window layers, short contexts) are cut evenly over all warps, which
+ *     has the shorter set-up.  PUZZLE_SCHED_CTA / PUZZLE_SCHED_WARP pin one or the other
+ *     (PUZZLE_SCHED_CTA needs batch <= 1024, else PUZZLE_ERR_UNSUPPORTED);
  *   workspace: device scratch of at least puzzle_decode_attn_workspace_bytes(...) bytes, 16-byte
  *     aligned, prepared once by puzzle_decode_attn_workspace_init; calls that share a workspace must
- *     not overlap on the GPU;
+ *     not overlap on the GPU.  Besides partials and counters it keeps the CTA speeds between calls:
+ *     they change how the next launch is cut, never its result beyond rounding;
  *   dev_status: optional int32 device word (see PUZZLE_DEV_*).
  * An empty context gives out = 0 and lse = sink (-inf without a sink). */
 PUZZLE_API puzzle_status puzzle_decode_attn(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
@@ -221,10 +246,17 @@ PUZZLE_API puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* des
  *     the process exits.  A batch and split choice whose
  *     puzzle_decode_attn_workspace_bytes exceeds that size is refused with
  *     PUZZLE_ERR_WORKSPACE and nothing is launched (balanced schedule: batch up
- *     to about 280; explicit splits: batch * num_splits up to about 500).
+ *     to about 280 on a 148-SM device; explicit splits: batch * num_splits up to
+ *     about 500).
  *   - The call allocates and frees nothing.  The first call on each device looks
- *     up the array's device address (with that device current); make that first
- *     call before starting any stream capture.
+ *     up the array's device address (with that device current).  Make that first
+ *     call at start-up: before any stream capture, and before the caller hands
+ *     out the device's remaining memory, because the driver reserves the
+ *     array's 8 MiB when it loads the library's device image, which can be as
+ *     late as this first call.  From the second call on, free device memory
+ *     does not change.
+ *   - Argument errors are reported before anything is enqueued, as for every
+ *     entry point: an invalid call neither clears nor touches the array.
  *   - All calls on a device share the one array.  Two calls that overlap on the
  *     GPU (different streams, no dependency between them) race on it and both
  *     results are undefined; order them.  The array keeps the previous call's
@@ -237,7 +269,10 @@ PUZZLE_API puzzle_status puzzle_decode_attn_static(const puzzle_layer_desc* desc
 
 /* Log-sum-exp merge of partial attention results that came from elsewhere
  * (e.g. context shards on other GPUs; puzzle_decode_attn merges its own
- * partials itself).  For every row r = (b, g):
+ * partials itself).  It is the second half of the split-KV pass of the
+ * KV-I/O-bound decode (paper, Section "Optimized Scenarios"); the paper does not
+ * define the merge: the formula is the exact recombination of softmax partials,
+ * with the per-head sink logit counted once.  For every row r = (b, g):
  *     M = max(sink_g, max_p lse_p),  Z = e^(sink_g - M) + sum_p e^(lse_p - M),
  *     out = sum_p e^(lse_p - M) o_p / Z,  lse_out = M + ln Z.
  *   part_o: float32 [batch][Hq][S][D];  part_lse: float32 [batch][Hq][S] (natural log; -inf = empty part);
@@ -247,7 +282,9 @@ PUZZLE_API puzzle_status puzzle_attn_merge(const float* part_o, const float* par
                                 const float* sinks, void* out, float* lse_out, int32_t batch, int32_t Hq,
                                 int32_t D, int32_t S, void* stream);
 
-/* puzzle_attn_merge over partials laid out with strides (in floats): part k of row r = b * Hq + g has
+/* puzzle_attn_merge (same passage, same formula) over partials laid out with strides (in floats), for the
+ * exchange step of a context-sharded layer (serving over 1..8 GPUs: paper, paragraph "Inference efficiency
+ * benchmarking"): part k of row r = b * Hq + g has
  * its D outputs at part_o + r * o_row_stride + k * o_part_stride and its lse at
  * part_lse[r * lse_row_stride + k * lse_part_stride].  An all-gather of per-device buffers
  * {o [batch][Hq][D], lse [batch][Hq]} is merged in place with o_row_stride = D,

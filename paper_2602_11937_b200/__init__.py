@@ -11,6 +11,9 @@ from .binding import (  # noqa: F401
     DEV_SEQ_TOO_LONG,
     DEV_WAIT_EXPIRED,
     STATIC_SCRATCH_BYTES,
+    SCHED_AUTO,
+    SCHED_CTA,
+    SCHED_WARP,
     KVView,
     LayerDesc,
     PuzzleError,

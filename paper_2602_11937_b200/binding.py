@@ -8,8 +8,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# PUZZLE_ATTN_LIB points the binding at another build of the same library (e.g. a tuning variant)
-_LIB_PATH = os.environ.get("PUZZLE_ATTN_LIB") or os.path.join(_HERE, "lib", "libpuzzle_attn.so")
+_LIB_PATH = os.path.join(_HERE, "lib", "libpuzzle_attn.so")
 _lib = None
 
 KV_FP8_E4M3 = 0
@@ -18,6 +17,7 @@ DEV_BAD_BLOCK = 1
 DEV_SEQ_TOO_LONG = 2
 DEV_WAIT_EXPIRED = 4
 STATIC_SCRATCH_BYTES = 8 << 20
+SCHED_AUTO, SCHED_CTA, SCHED_WARP = 0, -1, -2      # num_splits values that select the balanced schedule
 
 EXPORTS = (
     "puzzle_kv_amax_update",

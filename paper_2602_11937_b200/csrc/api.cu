@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/puzzle_attn.h: argument checks, TMA descriptor
 // encoding and kernel launches.  No allocation, no synchronisation, no state besides a launch counter.
+#include <algorithm>
 #include <atomic>
 #include <cstring>
 
@@ -102,8 +103,18 @@ size_t counter_bytes(int batch, int Hkv) {
   return (((size_t)batch * Hkv + cta_rate_words(grid_ctas())) * sizeof(int32_t) + 255) & ~(size_t)255;
 }
 
-// The balanced schedule runs on the CTA-balanced kernel when the batch fits its shared-memory schedule.
-bool use_cta_kernel(int batch, int num_splits) { return num_splits == 0 && batch <= kCtaMaxBatch; }
+// The balanced schedule runs on the CTA-balanced kernel when the batch fits its shared-memory schedule and the
+// launch can be large: with at most a few tiles per warp (window layers, short contexts) a launch is a chain of
+// latencies, which the warp-scheduled kernel's shorter set-up serves better.  The bound on the tiles comes from
+// what the host knows: the window, or the length of a block-table row.
+bool use_cta_kernel(const puzzle_layer_desc* d, const puzzle_kv_view* kv, int batch, int num_splits) {
+  if (num_splits == PUZZLE_SCHED_CTA) return true;
+  if (num_splits != 0 || batch > kCtaMaxBatch) return false;
+  const int tt = d->kv_dtype == PUZZLE_KV_FP8_E4M3 ? kTileFp8 : kTileBf16;
+  long long per_pair = ((long long)kv->max_blocks_per_seq * kBlock + tt - 1) / tt;
+  if (d->window > 0) per_pair = std::min<long long>(per_pair, (d->window + tt - 1) / tt + 1);
+  return per_pair * batch * d->num_kv_heads >= (long long)kCtaMinTilesPerCta * grid_ctas();
+}
 
 size_t workspace_floats(int batch, int Hkv, int num_splits, int kv_dtype) {
   size_t rows;
@@ -118,6 +129,22 @@ size_t workspace_floats(int batch, int Hkv, int num_splits, int kv_dtype) {
 }
 
 }  // namespace
+
+// Everything about a decode-attention call that the host can check, short of the workspace.
+puzzle_status check_decode_attn_args(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                     const void* out, int batch, int num_splits, bool tcgen05) {
+  puzzle_status st = check_desc(desc);
+  if (st != PUZZLE_OK) return st;
+  st = check_view(desc, kv, batch);
+  if (st != PUZZLE_OK) return st;
+  if (!q || !out) return PUZZLE_ERR_NULL;
+  if (num_splits < PUZZLE_SCHED_WARP || num_splits > 65536) return PUZZLE_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(q) & 7) || (reinterpret_cast<uintptr_t>(out) & 15)) return PUZZLE_ERR_SHAPE;
+  if (num_splits == PUZZLE_SCHED_CTA && (tcgen05 || batch > kCtaMaxBatch)) return PUZZLE_ERR_UNSUPPORTED;
+  if (tcgen05 && desc->kv_dtype != PUZZLE_KV_FP8_E4M3) return PUZZLE_ERR_UNSUPPORTED;   // that kernel reads E4M3 codes only
+  return PUZZLE_OK;
+}
+
 }  // namespace puzzle
 
 using namespace puzzle;
@@ -177,26 +204,22 @@ puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, const puzzl
 }
 
 size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits) {
-  if (check_desc(desc) != PUZZLE_OK || batch <= 0 || batch > kMaxBatch || num_splits < 0) return 0;
+  if (check_desc(desc) != PUZZLE_OK || batch <= 0 || batch > kMaxBatch || num_splits < PUZZLE_SCHED_WARP) return 0;
   return counter_bytes(batch, desc->num_kv_heads) +
-         workspace_floats(batch, desc->num_kv_heads, num_splits, desc->kv_dtype) * sizeof(float);
+         workspace_floats(batch, desc->num_kv_heads, num_splits > 0 ? num_splits : 0, desc->kv_dtype) * sizeof(float);
 }
 
 static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
                                       const float* sinks, void* out, float* lse_out, int32_t batch,
                                       int32_t num_splits, void* workspace, size_t workspace_bytes,
                                       int32_t* dev_status, void* stream, bool tcgen05, bool out_f32 = false) {
-  puzzle_status st = check_desc(desc);
+  puzzle_status st = check_decode_attn_args(desc, kv, q, out, batch, num_splits, tcgen05);
   if (st != PUZZLE_OK) return st;
-  st = check_view(desc, kv, batch);
-  if (st != PUZZLE_OK) return st;
-  if (!q || !out) return PUZZLE_ERR_NULL;
-  if (num_splits < 0 || num_splits > 65536) return PUZZLE_ERR_SHAPE;
-  if ((reinterpret_cast<uintptr_t>(q) & 7) || (reinterpret_cast<uintptr_t>(out) & 15)) return PUZZLE_ERR_SHAPE;
   const int Hkv = desc->num_kv_heads;
   const bool fp8 = desc->kv_dtype == PUZZLE_KV_FP8_E4M3;
   const size_t cbytes = counter_bytes(batch, Hkv);
-  const size_t pfloats = workspace_floats(batch, Hkv, num_splits, desc->kv_dtype);
+  const int splits = num_splits > 0 ? num_splits : 0;   // the kernels know explicit splits (S) and balanced (0)
+  const size_t pfloats = workspace_floats(batch, Hkv, splits, desc->kv_dtype);
   const size_t need = cbytes + pfloats * sizeof(float);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 15)) return PUZZLE_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -209,7 +232,6 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   DecodeParams P;
   std::memset(&P, 0, sizeof P);
   const int eb = fp8 ? 1 : 2;
-  if (tcgen05 && !fp8) return PUZZLE_ERR_UNSUPPORTED;   // the tensor-memory kernel reads E4M3 codes only
   const bool tc = tcgen05;
   const int row_bytes = tc ? 64 : 128;
   const int rows_per_block = kBlock * kHeadDim * eb / row_bytes;
@@ -235,7 +257,7 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   P.Hkv = Hkv;
   P.max_blocks_per_seq = kv->max_blocks_per_seq;
   P.window = desc->window;
-  P.num_splits = num_splits;
+  P.num_splits = splits;
   P.oob_row = (int)cache_rows;
   P.rows_per_block = rows_per_block;
   P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
@@ -243,7 +265,7 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   cudaError_t le;
   if (tc) {
     le = launch_decode_attn_tc(P, ctas, s, device_info().smem_limit + 2);
-  } else if (use_cta_kernel(batch, num_splits)) {
+  } else if (use_cta_kernel(desc, kv, batch, num_splits)) {
     le = launch_decode_attn_cta(P, fp8, ctas, s, device_info().smem_limit + 3);
   } else {
     le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);

@@ -6,6 +6,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include "../../include/puzzle_attn.h"
+
 namespace puzzle {
 
 struct alignas(64) DecodeParams {
@@ -52,6 +54,7 @@ constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
 // CTA slot in the workspace (after the arrival counters: a CTA counter, the buffer switch, two pad words, then two
 // float buffers of one speed per CTA) and are cut by the speeds the launch before them noted.
 constexpr int kCtaMaxBatch = 1024;
+constexpr int kCtaMinTilesPerCta = 64;   // below this bound on the tiles per CTA the warp-scheduled kernel is used
 constexpr int kCtaRateMinTiles = 256;
 inline size_t cta_rate_words(int ctas) { return 4 + 2 * (size_t)ctas; }
 
@@ -65,6 +68,10 @@ cudaError_t launch_decode_attn_cta(const DecodeParams& P, bool fp8, int ctas, cu
 // (one token), box = 16 rows, 64-byte swizzle; P.rows_per_block is 16 and P.oob_row counts such rows.
 cudaError_t launch_decode_attn_tc(const DecodeParams& P, int ctas, cudaStream_t s, int* smem_limit);
 int decode_attn_tc_workers_per_cta();
+
+// Host-visible argument checks of the decode-attention entry points (everything but the workspace).
+puzzle_status check_decode_attn_args(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                     const void* out, int batch, int num_splits, bool tcgen05);
 
 __global__ void attn_merge_kernel(const MergeParams P);
 

@@ -422,21 +422,20 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
 
 #pragma unroll 1
   for (;;) {
+    // the next tile's description is known since the tile was issued: a change of piece (its hand-over, the new
+    // query) is dealt with while the tile's bytes are still on their way
     int4 d0 = make_int4(0, 0, 0, -1), d1 = make_int4(0, 0, 0, 0);
-    const bool more = inflight > 0 && !failed;
+    const bool more = inflight > 0;
     if (more) {
-      if (!mbar_wait_bounded(bars + 8 * stage, phase)) {
-        failed = true;
-      } else {
-        --inflight;
-        d0 = lds128_volatile(desc_a + stage * sizeof(TileDesc));
-        d1 = lds128_volatile(desc_a + stage * sizeof(TileDesc) + 16);
-      }
+      d0 = lds128_volatile(desc_a + stage * sizeof(TileDesc));
+      d1 = lds128_volatile(desc_a + stage * sizeof(TileDesc) + 16);
     }
-    if (failed) break;
     if (d0.w != cur_k) {
       // ---- the piece changes (or nothing is left): hand this warp's share of the old piece over
       if (cur_k >= 0) {
+        // fetched now, used at the very end (only the warp that completes the piece needs them)
+        const float vs = P.v_scale && FP8 ? __ldg(P.v_scale + cur_kvh) : 1.f;
+        const float sink_g = P.sinks ? __ldg(P.sinks + cur_kvh * kGroup + g) : -INFINITY;
         float l_tot = st.l_run;
         l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
         l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
@@ -523,13 +522,12 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
           const int p = ctl.p_first + cur_k;
           const int nt = (cum[cur_b + 1] - cum[cur_b]) / P.Hkv;
           const int ps = cum[cur_b] + cur_kvh * nt;
-          int c_first;
-          const int count = ranges_of(bound, nC, ps, ps + nt, c_first);
-          const float vs = P.v_scale && FP8 ? P.v_scale[cur_kvh] : 1.f;
+          int c_first = blockIdx.x;
+          const int count = cur_total == nt ? 1 : ranges_of(bound, nC, ps, ps + nt, c_first);  // the whole pair is here
           if (count == 1) {
             const int head = cur_kvh * kGroup + g;
             const long long row_out = (long long)cur_b * (P.Hkv * kGroup) + head;
-            const float s2 = P.sinks ? P.sinks[head] * 1.4426950408889634f : -INFINITY;
+            const float s2 = sink_g * 1.4426950408889634f;
             const float M = fmaxf(l_tot > 0.f ? m : -INFINITY, s2);
             float f = 0.f, Z = 0.f;
             if (M != -INFINITY) {
@@ -579,6 +577,11 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
       st.reset();
     }
     if (!more) break;
+    if (!mbar_wait_bounded(bars + 8 * stage, phase)) {
+      failed = true;
+      break;
+    }
+    --inflight;
     const uint32_t kbase = pipe + stage * STAGE_BYTES;
     const uint32_t vbase = kbase + NB * BLOCK_BYTES;
     const int tok0 = d0.z * TT;
@@ -593,8 +596,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
     const int r = prod.template issue<BLOCK_BYTES>(ctl_a, P, cum, pc_a, rec_a, lane, kbase, bars + 8 * stage,
                                                    desc_a + stage * sizeof(TileDesc));
     if (r != 0) ++inflight;
-    if (r < 0) failed = true;
     if (++stage == NS) { stage = 0; phase ^= 1u; }
+    if (r < 0) { failed = true; break; }
   }
 
   // pairs without any visible key have no tile and hence no piece: zeros (lse = sink) from here

@@ -8,6 +8,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "decode_attn.cuh"
 
 namespace puzzle {
 namespace {
@@ -44,13 +45,15 @@ extern "C" puzzle_status puzzle_decode_attn_static(const puzzle_layer_desc* desc
                                                    int32_t batch, int32_t num_splits, int32_t* dev_status,
                                                    void* stream) {
   using namespace puzzle;
+  // argument errors first: an invalid call must not put the counter clear on the stream (it could zero the
+  // counters under a call that is still running on another stream)
+  puzzle_status st = check_decode_attn_args(desc, kv, q, out, batch, num_splits, false);
+  if (st != PUZZLE_OK) return st;
   const size_t need = puzzle_decode_attn_workspace_bytes(desc, batch, num_splits);
-  if (need == 0) {  // let the allocating entry point name the argument error (it fails before any launch)
-    return puzzle_decode_attn(desc, kv, q, sinks, out, lse_out, batch, num_splits, nullptr, 0, dev_status, stream);
-  }
+  if (need == 0) return PUZZLE_ERR_SHAPE;
   if (need > kStaticScratchBytes) return PUZZLE_ERR_WORKSPACE;
   void* scratch = nullptr;
-  puzzle_status st = scratch_address(&scratch);
+  st = scratch_address(&scratch);
   if (st != PUZZLE_OK) return st;
   // The array keeps whatever the previous call left.  Only the arrival counters must start at zero; a call
   // that ran to its end leaves them so, but one that was cut short does not, so they are cleared every time.

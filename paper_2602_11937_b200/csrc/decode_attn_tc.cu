@@ -21,7 +21,9 @@
 //    only when a tile exceeds it by more than 2^8.
 //  * At the end of a (sequence, KV head) run the group reads the accumulator, writes one float32 partial
 //    (o, lse); the worker whose partial completes a (sequence, KV head) merges all of them and stores bf16.
-//  Every wait is bounded; a wait that runs out sets PUZZLE_DEV_WAIT_EXPIRED, and every role leaves its loop.
+//  Every wait is bounded, the barrier of a group's softmax warps included (an mbarrier with a poll limit that
+//  also watches the abort flag, not a named barrier): a wait that runs out sets PUZZLE_DEV_WAIT_EXPIRED and the
+//  abort flag, and every role then leaves its loop, whichever warp of a group notices first.
 //
 //  Copies and MMAs are issued under an elect.sync predicate with the whole warp in the loop: inside an
 //  `if (lane == 0)` branch the compiler elects a lane and moves every operand to a uniform register per
@@ -65,6 +67,7 @@ struct GroupCtl {
   uint64_t p_full[2], pv_done[2];
   uint64_t verdict[2];     // the softmax warps have posted whether the reference maximum covers their rows
   uint64_t q_full;
+  uint64_t gsync;          // barrier of the group's softmax warps (one arrival per warp)
   float alpha[kGroup];     // logit scale per head in log2 units (k_scale and the query's power of two folded in)
   float xchg[4][kGroup];   // per-warp values exchanged inside the group (tile maxima, weight sums)
   int raise[2];            // by tile parity: some warp's rows exceed the reference by more than 2^8
@@ -95,7 +98,6 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(1 + g), "n"(32 * SW) : "memory"); }
 
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units), layout type
 // (0 = no swizzle, 4 = 64-byte swizzle), descriptor version 1.
@@ -187,6 +189,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
         c->raise[i] = 0;
       }
       mbar_init(smem_u32(&c->q_full), SW);
+      mbar_init(smem_u32(&c->gsync), SW);
     }
     C->abort = 0;
     fence_mbar_init();
@@ -370,11 +373,27 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
     const uint32_t td = tmem + g * kTmemCols + ((uint32_t)(32 * wq) << 16);
     int n = 0;
     bool dead = false;
+    // Barrier of the group's eight softmax warps on an mbarrier, so that it has a limit like every other wait: a
+    // warp that has left (its own wait ran out, or it saw the abort flag) lets the others run into the limit or
+    // see the flag, never wait for ever.  False: leave.
+    uint32_t gphase = 0;
+    auto group_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl->gsync));
+      bool ok = false;
+      for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(smem_u32(&ctl->gsync), gphase)) { ok = true; break; }
+        if (C->abort) break;
+      }
+      gphase ^= 1u;
+      if (!ok) { give_up(); dead = true; }
+      return ok;
+    };
     while (!dead && !C->abort && next_segment<TT>(cur, seg, P, cum, lens, w)) {
       if (seg.t == seg.t_end) {  // empty split (explicit schedule): weight zero
         if (gi < kGroup) P.part_lse[seg.prow + gi * seg.pstride] = -INFINITY;
         __threadfence();
-        group_sync(g);
+        if (!group_sync()) break;
         if (gi < 32) arrive_and_merge(P, seg.b, seg.kvh, cum, nW, lane);
         continue;
       }
@@ -419,7 +438,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
         }
       }
       fence_proxy_async();    // the query rows are read by the tensor core
-      group_sync(g);
+      if (!group_sync()) break;
       if (lane == 0) mbar_arrive(smem_u32(&ctl->q_full));
       float a_hi[4], a_lo[4], m_ref[4], l_run[4];
 #pragma unroll
@@ -503,7 +522,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
             for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, d));
             if (lane == 0) ctl->xchg[wq][H0 + i] = mx;
           }
-          group_sync(g);
+          if (!group_sync()) break;
           if (gi == 0) ctl->raise[b] = 0;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -532,7 +551,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
             tmem_wait_st();
             tc_fence_before();
           }
-          group_sync(g);   // xchg / raise may be rewritten only after everyone has read them
+          if (!group_sync()) break;   // xchg / raise may be rewritten only after everyone has read them
           weights();       // again, against the raised reference
         }
 #pragma unroll
@@ -570,7 +589,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
         for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(kFull, v, d);
         if (lane == 0) ctl->xchg[wq][H0 + i] = v;
       }
-      group_sync(g);
+      if (!group_sync()) break;
       {
         uint32_t o0[8], o1[8];   // terms 1, 2 and terms 3, 4 of this half's heads
         tmem_ld8(td + kO + 8 * hh, o0);
@@ -593,7 +612,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
         }
       }
       __threadfence();
-      group_sync(g);
+      if (!group_sync()) break;
       if (gi < 32) arrive_and_merge(P, seg.b, seg.kvh, cum, nW, lane);
     }
     // sequences without any visible key have no tile and hence no worker in the balanced schedule

@@ -99,6 +99,32 @@ def test_full_size_64k_context_split_sweep():
         case.attn_and_check(0, num_splits=s, rel=True, seed=s)
 
 
+def test_full_size_8k_context_full_and_window_layers():
+    """Batch 32, context 8192, paged: the full-attention layer and the 128-token window layer of the short-context
+    workload at its full size; the full layer is run twice on one workspace, so that the second launch is cut by
+    the CTA speeds the first one noted."""
+    w = synth.workload(2)
+    full = FullCase(w, 0)
+    full.append_and_check()
+    full.attn_and_check(0, seed=3, n_items=24)
+    P = full.P
+    d = full.desc(0)
+    ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(d, w.batch, 0), dtype=torch.uint8, device="cuda")
+    P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
+    outs = []
+    for _ in range(3):
+        o = torch.empty(w.batch, w.hq, w.head_dim, dtype=torch.bfloat16, device="cuda")
+        P.puzzle_decode_attn(d, full.view, full.q, full.sinks, o, None, workspace=ws, dev_status=full.status)
+        outs.append(o.float().cpu().numpy().astype(np.float64))
+    torch.cuda.synchronize()
+    assert int(full.status.item()) == 0
+    for o in outs[1:]:
+        assert np.all(np.abs(o - outs[0]) <= 2e-3 + 2.0 ** -7 * np.abs(outs[0]))
+    win = FullCase(w, 1)
+    win.append_and_check()
+    win.attn_and_check(128, seed=4, n_items=24)
+
+
 def test_full_size_ragged_stack_layers():
     """Batch 64, ragged contexts in [16K, 48K]: one cache, the three layer kinds of the 36-layer patterns."""
     case = FullCase(synth.workload(4), 1)

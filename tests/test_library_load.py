@@ -49,3 +49,20 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "_LIB_PATH", "/nonexistent/libpuzzle_attn.so")
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         binding.puzzle_launch_count()
+
+
+def test_static_entry_point_reports_argument_errors_before_touching_the_device():
+    """A NULL q (or out) is an argument error of puzzle_decode_attn_static that the host sees: it returns
+    PUZZLE_ERR_NULL without a CUDA call, so this runs without a GPU.  The cache pointers are never followed."""
+    from paper_2602_11937_b200 import binding
+    lib = binding._load()
+    desc = binding.layer_desc()
+    kv = binding.KVView()
+    kv.k_cache, kv.v_cache, kv.seq_lens = 0x1000, 0x2000, 0x3000
+    kv.num_blocks, kv.max_blocks_per_seq = 64, 16
+    kv.block_table, kv.k_scale, kv.v_scale = None, None, None
+    call = lambda q, out: lib.puzzle_decode_attn_static(ctypes.byref(desc), ctypes.byref(kv), q, None, out, None, 4, 0,
+                                                        None, None)
+    assert call(None, ctypes.c_void_p(0x5000)) == 1      # PUZZLE_ERR_NULL
+    assert call(ctypes.c_void_p(0x4000), None) == 1
+    assert call(ctypes.c_void_p(0x4004), ctypes.c_void_p(0x5000)) == 2   # q not 8-byte aligned: PUZZLE_ERR_SHAPE
