@@ -558,6 +558,87 @@ def run_stack(args):
         "dev_status": int(stack.status.item())}))
 
 
+# ------------------------------------------------- FP8 KV with and without scales ---
+
+def run_study(args):
+    """FP8 KV with calibrated scales, with scales rounded up to a power of two, and without scales (the three
+    settings of the paper's Section "KV Quantization"), on synthetic K/V streams: how many elements underflow to
+    zero, how many are clipped at +-448 (their nearest code would lie above it), the error of the dequantised values, and what that does to the attention
+    output.  Everything numeric runs in the library: the streams are quantised by puzzle_kv_append_tokens under
+    scales from puzzle_kv_amax_update / puzzle_kv_scales_from_amax, and the attention of the FP8 cache is compared
+    with the library's own bf16-cache path on the same samples.  Counting and averaging is done with torch.
+    Prints one JSON line per (stream, setting) and a markdown table."""
+    import paper_2602_11937_b200 as P
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    batch, n_tok = 4, 4096
+    w = synth.Workload("scale_study", 77, batch, n_tok, [0], paged=False)
+    nb = batch * w.blocks_per_seq
+    seq = torch.full((batch,), n_tok, dtype=torch.int32, device=dev)
+    q = synth.draw_q(w, 0, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    streams = [("gauss", 2.0 ** e) for e in (-8, -6, -4, -2, 0, 2, 4, 6, 8)] + [("heavy", 1.0), ("heavy", 2.0 ** -6),
+                                                                             ("heads", 1.0), ("heads", 2.0 ** -5)]
+    rows = []
+
+    def attention(desc, k_cache, v_cache, ks, vs):
+        view = P.kv_view(k_cache, v_cache, seq, max_blocks_per_seq=w.blocks_per_seq, k_scale=ks, v_scale=vs)
+        ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(desc, batch, 0), dtype=torch.uint8, device=dev)
+        P.puzzle_decode_attn_workspace_init(desc, batch, ws)
+        out = torch.empty(batch, w.hq, w.head_dim, dtype=torch.bfloat16, device=dev)
+        P.puzzle_decode_attn(desc, view, q, None, out, None, workspace=ws, dev_status=status)
+        return out.float()
+
+    for kind, sigma in streams:
+        xk = synth.draw_study_stream(kind, sigma, batch, n_tok, "k", dev)
+        xv = synth.draw_study_stream(kind, sigma, batch, n_tok, "v", dev)
+        # the comparison run: the same samples in a bf16 cache (cache layout [block][Hkv][16][D])
+        to_cache = lambda x: x.view(batch, w.blocks_per_seq, w.block, w.hkv, w.head_dim).permute(0, 1, 3, 2, 4) \
+            .reshape(nb, w.hkv, w.block, w.head_dim).contiguous()
+        ref = attention(P.layer_desc(kv_dtype=P.KV_BF16), to_cache(xk), to_cache(xv), None, None)
+        ref_max = float(ref.abs().max())
+        for setting in ("no scales", "amax/448", "amax/448 rounded up to 2^k"):
+            if setting == "no scales":
+                ks = torch.ones(w.hkv, device=dev)
+                vs = torch.ones(w.hkv, device=dev)
+            else:
+                ks = P.calibrate_scales([xk], w.hkv, pow2=setting.endswith("2^k"), device=dev)
+                vs = P.calibrate_scales([xv], w.hkv, pow2=setting.endswith("2^k"), device=dev)
+            desc = P.layer_desc()
+            kc = torch.zeros(nb, w.hkv, w.block, w.head_dim, dtype=torch.uint8, device=dev)
+            vc = torch.zeros_like(kc)
+            view = P.kv_view(kc, vc, seq, max_blocks_per_seq=w.blocks_per_seq, k_scale=ks, v_scale=vs)
+            P.puzzle_kv_append_tokens(desc, view, xk, xv, dev_status=status)
+            under = sat = 0.0
+            num = den = 0.0
+            for x, c, sc in ((xk, kc, ks), (xv, vc, vs)):
+                xf = to_cache(x).float()
+                code = c & 0x7F
+                y = xf / sc[None, :, None, None]
+                under += float(((code == 0) & (xf != 0)).float().mean()) / 2
+                sat += float((y.abs() >= 464).float().mean()) / 2      # nearest code would lie above 448
+                deq = c.view(torch.float8_e4m3fn).float() * sc[None, :, None, None]
+                num += float((deq - xf).double().square().sum())
+                den += float(xf.double().square().sum())
+            out = attention(desc, kc, vc, ks, vs)
+            err = float((out - ref).abs().max())
+            row = {"study": "fp8_kv_scales", "stream": kind, "sigma": sigma, "setting": setting,
+                   "underflow_frac": round(under, 6), "clipped_frac": round(sat, 6),
+                   "rms_rel_err": round((num / den) ** 0.5, 5), "attn_max_abs_err": round(err, 5),
+                   "attn_max_abs_err_over_max_out": round(err / max(ref_max, 1e-30), 5),
+                   "k_scale_head0": float(ks[0]), "dev_status": int(status.item())}
+            rows.append(row)
+            print(json.dumps(row))
+    print()
+    print("| stream | sigma | setting | underflow to 0 | clipped at 448 | RMS rel. error | attention max abs err / max abs out |")
+    print("|---|---|---|---|---|---|---|")
+    for r in rows:
+        print("| %s | 2^%d | %s | %.4f | %.4f | %.4f | %.4f |" % (
+            r["stream"], round(__import__("math").log2(r["sigma"])), r["setting"], r["underflow_frac"], r["clipped_frac"],
+            r["rms_rel_err"], r["attn_max_abs_err_over_max_out"]))
+
+
 # ------------------------------------------------------------ reference arm ---
 
 def run_reference(args):
@@ -628,6 +709,8 @@ def main():
     ap.add_argument("--layers", type=int, default=4, help="distinct layer caches rotated between steps")
     ap.add_argument("--stack", type=int, default=0, choices=[0, 4, 5],
                     help="instead of the headline run: one step of the 36-layer stack of workload 4 or 5")
+    ap.add_argument("--study", default=None, choices=["scales"],
+                    help="instead of the headline run: FP8 KV with, with power-of-two and without scales on synthetic streams")
     ap.add_argument("--pattern", default="parent", choices=["parent", "every4th", "selective"])
     ap.add_argument("--kv", default="fp8", choices=["fp8", "bf16"])
     ap.add_argument("--kernel", default="mma", choices=["mma", "tcgen05"],
@@ -643,7 +726,9 @@ def main():
     plan = launch_plan(args.gpus, os.environ)
     if plan[0] == "spawn":
         sys.exit(spawn_ranks(args.gpus))
-    if args.stack:
+    if args.study:
+        run_study(args)
+    elif args.stack:
         run_stack(args)
     elif args.impl == "reference":
         run_reference(args)

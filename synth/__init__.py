@@ -3,7 +3,10 @@
 This module only draws numbers and lays out block tables.  It holds none of
 the method's arithmetic (no quantisation, no attention, no scale rule), so the
 CPU oracle's tests and the CUDA path's tests can both draw their inputs here
-without sharing anything else.
+without sharing anything else.  (``synth.device`` is the one exception, and it
+says so: to fill gigabyte caches for full-size runs it casts drawn samples with
+PyTorch's own float8 type after dividing by amax/448; that prepares inputs,
+and both sides then read the resulting bytes.)
 
 The five workloads follow the decode-heavy serving scenarios (fixed-length
 prompts and generations such as 4K/4K and 64K/64K; a gpt-oss-style stack of 36
@@ -206,3 +209,29 @@ def logical_view(cache: torch.Tensor, table: Optional[torch.Tensor], b: int, n_t
     blocks = cache[idx.to(cache.device)]            # [nb][Hkv][16][D]
     seq = blocks.permute(0, 2, 1, 3).reshape(-1, cache.shape[1], cache.shape[3])
     return seq[:n_tokens]
+
+
+STUDY_KINDS = ("gauss", "heavy", "heads")
+
+
+def draw_study_stream(kind: str, sigma: float, batch: int, n_tokens: int, which: str = "k", device: str = "cpu",
+                      hkv: int = HKV, head_dim: int = HEAD_DIM, seed: int = SEED_BASE + 77) -> torch.Tensor:
+    """K or V samples for the scale study, bf16 [batch][n_tokens][Hkv][D].
+
+    gauss: N(0, sigma^2).  heavy: sigma times a Student-t draw with 3 degrees of freedom (rare large values, as
+    activation outliers are).  heads: N(0, (sigma * 2^(h - Hkv/2))^2) for KV head h, i.e. heads whose magnitudes
+    spread over 2^Hkv."""
+    g = _gen(seed, S_K if which == "k" else S_V, int(round(8 * (8 + torch.log2(torch.tensor(float(sigma))).item()))), device)
+    shape = (batch, n_tokens, hkv, head_dim)
+    z = torch.randn(shape, generator=g, device=device)
+    if kind == "gauss":
+        x = z * sigma
+    elif kind == "heavy":
+        chi = torch.randn((3,) + shape, generator=g, device=device).square().sum(0) / 3.0
+        x = z / chi.sqrt() * sigma
+    elif kind == "heads":
+        f = sigma * torch.pow(2.0, torch.arange(hkv, device=device, dtype=torch.float32) - hkv / 2)
+        x = z * f[None, None, :, None]
+    else:
+        raise ValueError(kind)
+    return x.to(torch.bfloat16)
