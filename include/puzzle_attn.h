@@ -231,6 +231,33 @@ PUZZLE_API puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* des
                                  int32_t num_splits, void* workspace, size_t workspace_bytes,
                                  int32_t* dev_status, void* stream);
 
+/* Decode attention for up to n_q new tokens per sequence in one call: the tokens of a multi-token decode step, or
+ * a chunk of a prompt after its bulk append (puzzle_kv_append_tokens), i.e. the input half of the paper's
+ * fixed-length scenarios (Section "Optimized Scenarios"), on full and window layers (Section "Window attention for
+ * long-context inference") over the FP8 cache (Section "KV Quantization").  Query token i of sequence b sits at
+ * position p = seq_lens[b] - q_lens[b] + i (seq_lens counted AFTER the append of all q_lens[b] tokens) and is one
+ * decode step of puzzle_decode_attn over the keys [p + 1 - min(W, p + 1), p] (all of [0, p] when window == 0): the
+ * mask is causal.  Pairs of query tokens share one pass over the cache tiles, so two tokens cost little more than
+ * one; the kernel is bound by KV bytes like the single-token one.
+ *   q: bf16 [batch][n_q][num_q_heads][head_dim], 8-byte aligned;  q_lens: int32 [batch] real tokens per sequence
+ *     (clamped to [0, n_q]), or NULL = n_q for all;  sinks as puzzle_decode_attn;
+ *   out: bf16 [batch][n_q][num_q_heads][head_dim], 16-byte aligned: rows i < q_lens[b] are written, the others left
+ *     as they are;  lse_out: float32 [batch][n_q][num_q_heads] or NULL;
+ *   workspace: at least puzzle_decode_attn_tokens_workspace_bytes(desc, batch, n_q) bytes, 16-byte aligned,
+ *     prepared once by puzzle_decode_attn_tokens_workspace_init (zero-fills its arrival counters; every completed
+ *     call leaves them at zero); not to be shared with calls that overlap on the GPU;
+ *   a token whose position would be negative (q_lens[b] > seq_lens[b]) sees no key: out = 0, lse = sink.
+ * FP8 caches only (PUZZLE_ERR_UNSUPPORTED for bf16: give puzzle_decode_attn one batch row per query token instead);
+ * batch * ceil(n_q / 2) <= 8192 (PUZZLE_ERR_SHAPE).  Errors and dev_status as puzzle_decode_attn. */
+PUZZLE_API size_t puzzle_decode_attn_tokens_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t n_q);
+PUZZLE_API puzzle_status puzzle_decode_attn_tokens_workspace_init(const puzzle_layer_desc* desc, int32_t batch,
+                                                                  int32_t n_q, void* workspace, size_t workspace_bytes,
+                                                                  void* stream);
+PUZZLE_API puzzle_status puzzle_decode_attn_tokens(const puzzle_layer_desc* desc, const puzzle_kv_view* kv,
+                                                   const void* q, const int32_t* q_lens, const float* sinks, void* out,
+                                                   float* lse_out, int32_t batch, int32_t n_q, void* workspace,
+                                                   size_t workspace_bytes, int32_t* dev_status, void* stream);
+
 /* Size of the scratch array built into the library for puzzle_decode_attn_static. */
 #define PUZZLE_STATIC_SCRATCH_BYTES (8u << 20)
 

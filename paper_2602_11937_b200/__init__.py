@@ -27,6 +27,9 @@ from .binding import (  # noqa: F401
     puzzle_decode_attn_partial,
     puzzle_decode_attn_static,
     puzzle_decode_attn_tcgen05,
+    puzzle_decode_attn_tokens,
+    puzzle_decode_attn_tokens_workspace_bytes,
+    puzzle_decode_attn_tokens_workspace_init,
     puzzle_decode_attn_workspace_bytes,
     puzzle_decode_attn_workspace_init,
     puzzle_hbm_read_probe,

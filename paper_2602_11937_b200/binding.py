@@ -30,6 +30,9 @@ EXPORTS = (
     "puzzle_decode_attn_tcgen05",
     "puzzle_decode_attn_static",
     "puzzle_decode_attn_partial",
+    "puzzle_decode_attn_tokens",
+    "puzzle_decode_attn_tokens_workspace_bytes",
+    "puzzle_decode_attn_tokens_workspace_init",
     "puzzle_attn_merge",
     "puzzle_attn_merge_strided",
     "puzzle_hbm_read_probe",
@@ -96,6 +99,13 @@ def _load():
         lib.puzzle_decode_attn_static.restype = ctypes.c_int
         lib.puzzle_decode_attn_static.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp,
                                                   i32, i32, vp, vp]
+        lib.puzzle_decode_attn_tokens_workspace_bytes.restype = sz
+        lib.puzzle_decode_attn_tokens_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32, i32]
+        lib.puzzle_decode_attn_tokens_workspace_init.restype = ctypes.c_int
+        lib.puzzle_decode_attn_tokens_workspace_init.argtypes = [ctypes.POINTER(LayerDesc), i32, i32, vp, sz, vp]
+        lib.puzzle_decode_attn_tokens.restype = ctypes.c_int
+        lib.puzzle_decode_attn_tokens.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp, vp,
+                                                  i32, i32, vp, sz, vp, vp]
         lib.puzzle_attn_merge.restype = ctypes.c_int
         lib.puzzle_attn_merge.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
         lib.puzzle_hbm_read_probe.restype = ctypes.c_int
@@ -210,6 +220,32 @@ def puzzle_kv_append_tokens(desc: LayerDesc, view: KVView, k_new: torch.Tensor, 
                                            _p(v_new, torch.bfloat16, "v_new"), _p(new_lens, torch.int32, "new_lens"),
                                            batch, n_new, _p(dev_status, torch.int32), _stream(stream)),
            "puzzle_kv_append_tokens")
+
+
+def puzzle_decode_attn_tokens_workspace_bytes(desc: LayerDesc, batch: int, n_q: int) -> int:
+    return int(_load().puzzle_decode_attn_tokens_workspace_bytes(ctypes.byref(desc), int(batch), int(n_q)))
+
+
+def puzzle_decode_attn_tokens_workspace_init(desc: LayerDesc, batch: int, n_q: int, workspace: torch.Tensor,
+                                             stream=None) -> None:
+    _check(_load().puzzle_decode_attn_tokens_workspace_init(ctypes.byref(desc), int(batch), int(n_q), _p(workspace),
+                                                            workspace.numel() * workspace.element_size(),
+                                                            _stream(stream)), "puzzle_decode_attn_tokens_workspace_init")
+
+
+def puzzle_decode_attn_tokens(desc: LayerDesc, view: KVView, q: torch.Tensor, sinks: Optional[torch.Tensor],
+                              out: torch.Tensor, lse_out: Optional[torch.Tensor] = None,
+                              q_lens: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                              dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """q, out: bf16 [batch][n_q][Hq][D]; q_lens: int32 [batch] or None; see include/puzzle_attn.h."""
+    if workspace is None:
+        raise ValueError("a workspace tensor is required (see puzzle_decode_attn_tokens_workspace_bytes)")
+    batch, n_q = q.shape[0], q.shape[1]
+    _check(_load().puzzle_decode_attn_tokens(ctypes.byref(desc), ctypes.byref(view), _p(q, torch.bfloat16, "q"),
+                                             _p(q_lens, torch.int32, "q_lens"), _p(sinks, torch.float32, "sinks"),
+                                             _p(out, torch.bfloat16, "out"), _p(lse_out, torch.float32, "lse_out"),
+                                             batch, n_q, _p(workspace), workspace.numel() * workspace.element_size(),
+                                             _p(dev_status, torch.int32), _stream(stream)), "puzzle_decode_attn_tokens")
 
 
 def puzzle_decode_attn_workspace_bytes(desc: LayerDesc, batch: int, num_splits: int = 0) -> int:

@@ -33,7 +33,7 @@ EncodeTiledFn encode_tiled() {
 struct DeviceInfo {
   int sm_count = 0;
   // per split-KV kernel (warp-scheduled FP8, bf16; tensor-memory FP8; CTA-balanced FP8, bf16); 0 = not raised yet
-  int smem_limit[5] = {0, 0, 0, 0, 0};
+  int smem_limit[6] = {0, 0, 0, 0, 0, 0};   // [5]: the multi-token kernel
 };
 DeviceInfo& device_info() {
   static DeviceInfo info[64];
@@ -298,6 +298,76 @@ puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* desc, const pu
   if (!lse_part) return PUZZLE_ERR_NULL;
   return decode_attn_impl(desc, kv, q, nullptr, o_part, lse_part, batch, num_splits, workspace, workspace_bytes,
                           dev_status, stream, false, true);
+}
+
+static size_t tokens_counter_bytes(int batch, int n_q, int Hkv) {
+  return (decode_attn_tokens_counters(batch, n_q, Hkv) * sizeof(int32_t) + 255) & ~(size_t)255;
+}
+
+size_t puzzle_decode_attn_tokens_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t n_q) {
+  if (check_desc(desc) != PUZZLE_OK || batch <= 0 || n_q <= 0 || (long long)batch * ((n_q + 1) / 2) > kTokMaxRows)
+    return 0;
+  return tokens_counter_bytes(batch, n_q, desc->num_kv_heads) +
+         decode_attn_tokens_partial_rows(grid_ctas(), batch, n_q, desc->num_kv_heads) * (kHeadDim + 1) * sizeof(float);
+}
+
+puzzle_status puzzle_decode_attn_tokens_workspace_init(const puzzle_layer_desc* desc, int32_t batch, int32_t n_q,
+                                                       void* workspace, size_t workspace_bytes, void* stream) {
+  puzzle_status st = check_desc(desc);
+  if (st != PUZZLE_OK) return st;
+  if (batch <= 0 || n_q <= 0 || (long long)batch * ((n_q + 1) / 2) > kTokMaxRows) return PUZZLE_ERR_SHAPE;
+  const size_t cbytes = tokens_counter_bytes(batch, n_q, desc->num_kv_heads);
+  if (!workspace || workspace_bytes < cbytes || (reinterpret_cast<uintptr_t>(workspace) & 15))
+    return PUZZLE_ERR_WORKSPACE;
+  return cudaMemsetAsync(workspace, 0, cbytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? PUZZLE_OK
+                                                                                                  : PUZZLE_ERR_CUDA;
+}
+
+puzzle_status puzzle_decode_attn_tokens(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
+                                        const int32_t* q_lens, const float* sinks, void* out, float* lse_out,
+                                        int32_t batch, int32_t n_q, void* workspace, size_t workspace_bytes,
+                                        int32_t* dev_status, void* stream) {
+  puzzle_status st = check_decode_attn_args(desc, kv, q, out, batch, 0, false);
+  if (st != PUZZLE_OK) return st;
+  if (n_q <= 0 || (long long)batch * ((n_q + 1) / 2) > kTokMaxRows) return PUZZLE_ERR_SHAPE;
+  if (desc->kv_dtype != PUZZLE_KV_FP8_E4M3) return PUZZLE_ERR_UNSUPPORTED;   // the bf16 cache goes one row per token
+  const int Hkv = desc->num_kv_heads;
+  const size_t need = puzzle_decode_attn_tokens_workspace_bytes(desc, batch, n_q);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 15)) return PUZZLE_ERR_WORKSPACE;
+  const size_t cbytes = tokens_counter_bytes(batch, n_q, Hkv);
+  const size_t rows = decode_attn_tokens_partial_rows(grid_ctas(), batch, n_q, Hkv);
+  DecodeParams P;
+  std::memset(&P, 0, sizeof P);
+  const long long cache_rows = kv->num_blocks * Hkv * (long long)(kBlock * kHeadDim / 128);
+  if (!make_cache_map(&P.tmK, kv->k_cache, cache_rows, 1) || !make_cache_map(&P.tmV, kv->v_cache, cache_rows, 1))
+    return PUZZLE_ERR_CUDA;
+  P.q = static_cast<const __nv_bfloat16*>(q);
+  P.block_table = kv->block_table;
+  P.seq_lens = kv->seq_lens;
+  P.k_scale = kv->k_scale;
+  P.v_scale = kv->v_scale;
+  P.part_o = reinterpret_cast<float*>(static_cast<char*>(workspace) + cbytes);
+  P.part_lse = P.part_o + rows * kHeadDim;
+  P.counters = static_cast<int32_t*>(workspace);
+  P.sinks = sinks;
+  P.out = static_cast<__nv_bfloat16*>(out);
+  P.lse_out = lse_out;
+  P.dev_status = dev_status;
+  P.num_blocks = kv->num_blocks;
+  P.batch = batch;
+  P.Hkv = Hkv;
+  P.max_blocks_per_seq = kv->max_blocks_per_seq;
+  P.window = desc->window;
+  P.n_q = n_q;
+  P.q_lens = q_lens;
+  P.oob_row = (int)cache_rows;
+  P.rows_per_block = kBlock * kHeadDim / 128;
+  P.sm_scale_log2e = desc->sm_scale * 1.4426950408889634f;
+  if (launch_decode_attn_tokens(P, grid_ctas(), static_cast<cudaStream_t>(stream), device_info().smem_limit + 5) !=
+      cudaSuccess)
+    return PUZZLE_ERR_CUDA;
+  count_launch();
+  return PUZZLE_OK;
 }
 
 puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_desc* desc, int32_t batch, void* workspace,

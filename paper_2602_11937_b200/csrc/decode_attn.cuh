@@ -29,6 +29,8 @@ struct alignas(64) DecodeParams {
   long long num_blocks;
   int batch, Hkv, max_blocks_per_seq, window;
   int num_splits;  // 0 = balanced schedule
+  int n_q;         // multi-token kernel: query tokens per sequence in q / out ([batch][n_q][Hq][D]); else unused
+  const int32_t* q_lens;  // multi-token kernel: real query tokens per sequence [batch], or null (= n_q)
   int oob_row;     // a row coordinate outside the tensor maps: loads from it return zeros
   int rows_per_block;  // tensor-map rows (128 bytes each) per (block, KV head): 8 (FP8) or 16 (bf16)
   float sm_scale_log2e;
@@ -64,6 +66,13 @@ cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaSt
 // The CTA-balanced kernel (balanced schedule only, batch <= kCtaMaxBatch).  Its partial row blocks: one per
 // (CTA, pair) meeting, ctas + batch*Hkv at most.
 cudaError_t launch_decode_attn_cta(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit);
+// The multi-token kernel (FP8 cache, balanced schedule): P.n_q, P.q_lens set; P.counters has one word per
+// (sequence, token pair, KV head); partial rows: decode_attn_tokens_partial_rows(...).
+cudaError_t launch_decode_attn_tokens(const DecodeParams& P, int ctas, cudaStream_t s, int* smem_limit);
+size_t decode_attn_tokens_partial_rows(int ctas, int batch, int n_q, int Hkv);
+size_t decode_attn_tokens_counters(int batch, int n_q, int Hkv);
+constexpr int kTokMaxRows = 8192;   // (sequence, token pair) rows its shared-memory schedule holds
+
 // The tensor-memory (tcgen05) kernel for the FP8 cache.  Its tensor maps view the cache as rows of 64 bytes
 // (one token), box = 16 rows, 64-byte swizzle; P.rows_per_block is 16 and P.oob_row counts such rows.
 cudaError_t launch_decode_attn_tc(const DecodeParams& P, int ctas, cudaStream_t s, int* smem_limit);

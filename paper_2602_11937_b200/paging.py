@@ -54,7 +54,9 @@ def multi_token_args(seq_lens: torch.Tensor, block_table, n_q: int, max_blocks_p
     padding and get length 0 (output 0).  Pass q as ``[batch * n_q][Hq][D]``.
 
     The n_q rows of a sequence read the same cache blocks at about the same time (they are neighbours in the
-    balanced schedule), so the repeats are served by L2 rather than HBM."""
+    balanced schedule), so the repeats are served by L2 rather than HBM.  For FP8 caches
+    ``puzzle_decode_attn_tokens`` does the same job faster (pairs of query tokens share one pass over the tiles);
+    this form remains for bf16 caches and as a second way to the same result."""
     batch = seq_lens.shape[0]
     dev = seq_lens.device
     L = seq_lens.to(torch.int64)[:, None]

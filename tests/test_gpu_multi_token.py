@@ -87,3 +87,64 @@ def test_multi_token_causal_attention(window, kernel):
                                     case["sinks"], window, case["sm_scale"])
         assert_close(got[:, i], ref.reshape(w.batch, w.hq, w.head_dim), "query row %d, W=%d" % (i, window))
         assert not got[~real, i].any()                 # padding rows and absent queries give zeros
+
+
+@pytest.mark.parametrize("n_q", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("window", [0, 100])
+def test_tokens_kernel_shares_tiles_between_query_tokens(window, n_q):
+    """puzzle_decode_attn_tokens (pairs of query tokens on one pass over the tiles) against the oracle's
+    single-token step at every query position: ragged numbers of new tokens, sequences shorter than a tile, one
+    with no query, contexts that span many workers."""
+    import paper_2602_11937_b200 as P
+    from gpu_helpers import DeviceCase, assert_close
+    w = synth.Workload("tokq", 1, 6, 3000, [0], paged=True)
+    lens_after = np.array([3000, 2, 5, 333, 129, 1900], dtype=np.int32)
+    q_lens = np.minimum(np.array([n_q, 2, 5, 3, 0, n_q - 1 if n_q > 1 else 1], dtype=np.int32), n_q)
+    case = make_case(w, seq_lens=lens_after)
+    dev = DeviceCase(case)
+    k, v, q = _chunk(case, n_q, 50 + n_q)
+    ql_dev = torch.from_numpy(q_lens).cuda()
+    d = dev.desc(window)
+    P.puzzle_kv_append_tokens(d, dev.view(), k.cuda(), v.cuda(), ql_dev, dev_status=dev.status)
+    _oracle_append_chunk(case, lens_after, q_lens, k, v)
+    ws = torch.empty(P.puzzle_decode_attn_tokens_workspace_bytes(d, w.batch, n_q), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    P.puzzle_decode_attn_tokens_workspace_init(d, w.batch, n_q, ws)
+    for call in range(2):          # the second call finds the counters as the first one left them
+        out = torch.full((w.batch, n_q, w.hq, w.head_dim), 7.0, dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((w.batch, n_q, w.hq), 7.0, dtype=torch.float32, device="cuda")
+        P.puzzle_decode_attn_tokens(d, dev.view(), q.cuda(), dev.sinks, out, lse, q_lens=ql_dev, workspace=ws,
+                                    dev_status=dev.status)
+        torch.cuda.synchronize()
+        assert int(dev.status.item()) == 0
+        got = out.float().cpu().numpy().astype(np.float64)
+        got_lse = lse.cpu().numpy().astype(np.float64)
+        for i in range(n_q):
+            real = i < q_lens
+            step_lens = np.where(real, lens_after - q_lens + i + 1, 0).astype(np.int32)
+            ref, ref_lse = oracle.decode_attn(case["k_cache"], case["v_cache"], case["kv_dtype"], case["table"],
+                                              w.blocks_per_seq, step_lens, case["k_scale"], case["v_scale"],
+                                              bf16_bits(q[:, i].contiguous()), case["sinks"], window, case["sm_scale"])
+            ref = ref.reshape(w.batch, w.hq, w.head_dim)
+            assert_close(got[real, i], ref[real], "query row %d, W=%d, n_q=%d, call %d" % (i, window, n_q, call))
+            assert np.all(np.abs(got_lse[real, i] - ref_lse.reshape(w.batch, w.hq)[real]) <= 2e-3)
+            assert np.all(got[~real, i] == 7.0) and np.all(got_lse[~real, i] == 7.0)     # rows without a query: untouched
+
+
+def test_tokens_kernel_argument_errors():
+    import paper_2602_11937_b200 as P
+    from gpu_helpers import DeviceCase
+    w = synth.Workload("tokerr", 1, 2, 64, [0], paged=True)
+    dev = DeviceCase(make_case(w))
+    q = torch.zeros(2, 2, 64, 64, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(q)
+    ws = torch.zeros(P.puzzle_decode_attn_tokens_workspace_bytes(dev.desc(), 2, 2), dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.PuzzleError) as e:
+        P.puzzle_decode_attn_tokens(dev.desc(), dev.view(), q, None, out, workspace=ws[:256])
+    assert e.value.code == 4
+    bf = P.layer_desc(kv_dtype=P.KV_BF16)
+    with pytest.raises(P.PuzzleError) as e:
+        P.puzzle_decode_attn_tokens(bf, dev.view(), q, None, out, workspace=ws)
+    assert e.value.code == 3
+    assert P.puzzle_decode_attn_tokens_workspace_bytes(dev.desc(), 8192, 4) == 0      # too many rows
+    torch.cuda.synchronize()
