@@ -53,6 +53,8 @@ struct alignas(16) CtaCtl {
   long long t0;               // clock at kernel entry
   int warps_left;             // warps still running: the last one notes the CTA's speed
   int use_rates;              // this launch is large enough to note (and use) CTA speeds
+  int4 seed[2];               // the pair the range starts in, as a PairCache record: every warp starts from it
+  int first_n, pad[3];        // > 0: warp w's first claim is the first_n tiles from lo + w * first_n (no counter involved)
 };
 
 // Per-warp memory of the pair its last claim fell into (most claims fall into the same one again).  Two int4.
@@ -277,6 +279,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
   int* pk_key = reinterpret_cast<int*>(sp);                               sp += kPieceSlots * sizeof(int);
   int* pk_done = reinterpret_cast<int*>(sp);                              sp += kPieceSlots * sizeof(int);
   CtaCtl& ctl = *reinterpret_cast<CtaCtl*>(sp);                           sp += sizeof(CtaCtl);
+  static_assert(sizeof(CtaCtl) % 16 == 0, "the arrays behind it stay aligned");
   const uint32_t ctl_a = smem_u32(&ctl);
   int* bound = reinterpret_cast<int*>(sp);                                sp += ((nC + 1 + 3) & ~3) * sizeof(int);
   int* share = reinterpret_cast<int*>(sp);                                sp += ((nC + 1 + 3) & ~3) * sizeof(int);
@@ -310,13 +313,21 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
   // one warp turns the noted speeds into cumulative shares (fixed point, 4096 = the mean speed); without a full set
   // of speeds every CTA gets the same share
   if (warp == 1) {
-    const int ep = *reinterpret_cast<const volatile int*>(epoch_p) & 1;
-    float r[8];
+    // both buffers are fetched together with the switch that names the valid one: one round trip, not two
+    const int ep_word = __ldcg(epoch_p);
+    float r[8], r_other[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int cc = i * 32 + lane;
+      const bool on = cc < nC && i * 32 < nC;
+      r[i] = on ? __ldcg(rates + cc) : -1.f;
+      r_other[i] = on ? __ldcg(rates + nC + cc) : -1.f;
+    }
     float sum = 0.f, mn = 1e30f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int cc = i * 32 + lane;
-      r[i] = cc < nC && i * 32 < nC ? __ldcg(rates + ep * nC + cc) : -1.f;
+      if (ep_word & 1) r[i] = r_other[i];
       if (cc < nC) { sum += r[i]; mn = fminf(mn, r[i]); }
     }
 #pragma unroll
@@ -378,23 +389,34 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
       return x > 0 ? snap_cut(cum, P.batch, P.Hkv, x, snap) : 0;
     };
     for (int i = threadIdx.x; i <= nC; i += blockDim.x) bound[i] = boundary(i);
-    // two threads of otherwise idle warps work out this CTA's own range at the same time
+    // one thread of an otherwise idle warp works out this CTA's own range at the same time, the pair it starts in
+    // (every warp's first claim falls into it) and, when the first chunk of all NW warps lies inside that pair, hands
+    // those chunks out right here: twelve warps that start together would otherwise retry each other's
+    // compare-and-swap
     if (threadIdx.x == 32 * (NW - 1)) {
-      const int lo_c = boundary(blockIdx.x);
-      ctl.lo = ctl.pos = lo_c;
-      int pf = 0;  // the pair the range starts in (unused when the range is empty)
-      if (lo_c < T) {
+      const int lo_c = boundary(blockIdx.x), end_c = boundary(blockIdx.x + 1);
+      int pf = 0, first_n = 0;
+      int4 s0 = make_int4(0, 0, 0, 0), s1 = make_int4(0, 0, 0, 0);
+      if (lo_c < end_c) {
         const int b = seq_of(cum, P.batch, lo_c);
-        pf = b * P.Hkv + (lo_c - cum[b]) / ((cum[b + 1] - cum[b]) / P.Hkv);
+        const SeqTiles q = seq_tiles<TT>(P, b);
+        const int kvh = (lo_c - cum[b]) / q.nt;
+        pf = b * P.Hkv + kvh;
+        s0 = make_int4(cum[b] + kvh * q.nt, cum[b] + (kvh + 1) * q.nt, b, kvh);
+        s1 = make_int4(q.tlo, q.L, q.lo, 0);
+        const int c0 = max(1, min(kMaxChunk, (end_c - lo_c) >> 4));
+        if (min(s0.y, end_c) - lo_c >= NW * c0) first_n = c0;
       }
+      ctl.lo = lo_c;
+      ctl.end = end_c;
+      ctl.pos = lo_c + NW * first_n;
       ctl.p_first = pf;
-    }
-    if (threadIdx.x == 32 * (NW - 2)) {
-      ctl.end = boundary(blockIdx.x + 1);
+      ctl.seed[0] = s0;
+      ctl.seed[1] = s1;
+      ctl.first_n = first_n;
       ctl.warps_left = NW;
       ctl.use_rates = large ? 1 : 0;
     }
-    if (lane == 0) sts128(pc_a, make_int4(0, 0, 0, 0));
   }
   __syncthreads();
 
@@ -402,7 +424,23 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
   lo.init(lane);
 
   ClaimProducer<TT> prod;
-  bool failed = !prod.claim(ctl_a, P, cum, pc_a, rec_a, lane);
+  bool failed = false;
+  {
+    const int4 s0 = ctl.seed[0], s1 = ctl.seed[1];
+    const int first_n = ctl.first_n;
+    if (lane == 0) {
+      sts128(pc_a, s0);
+      sts128(pc_a + 16, s1);
+    }
+    if (first_n > 0) {  // this warp's share of the range's first tiles: the claim record written in place
+      const int pos = ctl.lo + warp * first_n;
+      prod.d.b = s0.z; prod.d.kvh = s0.w; prod.d.t = s1.x + (pos - s0.x); prod.d.k = 0;
+      prod.d.total = min(s0.y, ctl.end) - max(s0.x, ctl.lo); prod.d.L = s1.y; prod.d.lo = s1.z; prod.d.n = first_n;
+    } else {
+      __syncwarp();
+      failed = !prod.claim(ctl_a, P, cum, pc_a, rec_a, lane);
+    }
+  }
   prod.lookup(P, lane);
   int inflight = 0;
 #pragma unroll 1

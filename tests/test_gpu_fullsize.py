@@ -125,6 +125,50 @@ def test_full_size_8k_context_full_and_window_layers():
     win.attn_and_check(128, seed=4, n_items=24)
 
 
+def test_cta_speeds_change_the_cut_not_the_result():
+    """The CTA-balanced kernel cuts a large launch by the speed words that earlier launches left in the workspace.
+    Whatever those words hold (here: noise, huge and tiny values, negative ones, NaN and infinity patterns), the
+    result stays within the parity bound: they only move the cuts between CTAs."""
+    w = synth.workload(2)                    # batch 32, context 8192: 221 tiles per CTA ...
+    w.batch, w.context = 24, 16384           # ... made 24 x 16384: 332 tiles per CTA, above the size at which speeds are used
+    case = FullCase(w, 0)
+    case.append_and_check()
+    P = case.P
+    d = case.desc(0)
+    nbytes = P.puzzle_decode_attn_workspace_bytes(d, w.batch, P.SCHED_CTA)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
+    words = ws.view(torch.int32)
+    first = w.batch * w.hkv + 4               # after the arrival counters, the CTA counter, the switch and two pad words
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    rng = np.random.default_rng(5)
+    hk, hv = case.host
+    items = [(int(rng.integers(w.batch)), int(rng.integers(w.hq))) for _ in range(12)]
+    ref, _ = oracle.decode_attn(hk, hv, case.kv_dtype, _host(case.d["table"]), w.blocks_per_seq, case.lens_host,
+                                _host(case.d["k_scale"]), _host(case.d["v_scale"]), bf16_bits(case.q), _host(case.sinks),
+                                0, w.head_dim ** -0.5, items=items)
+    fills = [None,
+             lambda n: torch.from_numpy(rng.uniform(0.001, 10.0, n).astype(np.float32)),
+             lambda n: torch.from_numpy(rng.standard_normal(n).astype(np.float32)),
+             lambda n: torch.from_numpy(rng.integers(-2 ** 31, 2 ** 31 - 1, n).astype(np.int32)).view(torch.float32),
+             lambda n: torch.full((n,), float("inf")),
+             lambda n: torch.full((n,), 1e-30)]
+    for fill in fills:
+        if fill is not None:
+            words[first:first + 2 * n_sm] = fill(2 * n_sm).view(torch.int32).cuda()
+        for _ in range(2):                    # the second launch is cut by what the first one noted on top of it
+            out = torch.full((w.batch, w.hq, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+            P.puzzle_decode_attn(d, case.view, case.q, case.sinks, out, None, num_splits=P.SCHED_CTA, workspace=ws,
+                                 dev_status=case.status)
+            torch.cuda.synchronize()
+            assert int(case.status.item()) == 0
+            got_all = out.float().cpu().numpy().astype(np.float64)
+            assert np.isfinite(got_all).all()
+            got = np.stack([got_all[b, h] for b, h in items])
+            assert_close(got, ref, "speed words: %s" % ("zero" if fill is None else "filled"))
+    assert not words[: w.batch * w.hkv + 1].any()      # arrival counters and the CTA counter are back at zero
+
+
 def test_full_size_ragged_stack_layers():
     """Batch 64, ragged contexts in [16K, 48K]: one cache, the three layer kinds of the 36-layer patterns."""
     case = FullCase(synth.workload(4), 1)
