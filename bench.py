@@ -478,11 +478,11 @@ def cpu_baseline(w, layer, seq_lens_host, q, sinks, window, pairs: int = 128):
 # headline workload, from the one-launch `ncu --set full` capture summarised under profiles/; valid only for
 # the kernel sources it was taken from, so it is tied to their hash and reported as null once they change.
 NCU_CAPTURE = {
-    "source": "profiles/decode_attn_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
+    "source": "profiles/decode_attn_cta_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "b761b1d7f16384a72e8e4be46a8eb5f45977dbdbd6f9aa513875ae08bfdf039e",
-    "dram_bytes_per_launch": 1075472000 + 4413440,
+    "sha256": "970252cbcf07718876e513bb5d164475e0d38782661df01c3183f0be80bb7262",
+    "dram_bytes_per_launch": 1075474000 + 4500480,
 }
 
 
