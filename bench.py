@@ -481,7 +481,7 @@ NCU_CAPTURE = {
     "source": "profiles/decode_attn_cta_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "970252cbcf07718876e513bb5d164475e0d38782661df01c3183f0be80bb7262",
+    "sha256": "8f8215f3fdb8f28113d89312ca0ae20a4b9f0f420330ff720ac8a8aab48da05e",
     "dram_bytes_per_launch": 1075474000 + 4500480,
 }
 

@@ -11,7 +11,7 @@
 //    and window layers included) is cut into one contiguous range per CTA.  Inside a CTA the twelve warps do not
 //    own fixed shares: a warp takes the next tiles of the CTA's range (up to 16, fewer towards its end) with one
 //    compare-and-swap on a shared-memory counter whenever its own TMA ring runs dry, so the warps of an SM finish
-//    together.
+//    together.  (Only the very first chunk of every warp is fixed at set-up, when all twelve lie in one pair.)
 //  * On large launches every CTA notes how many tiles per cycle it managed; the next large launch on the same
 //    workspace cuts the ranges in proportion to those speeds (clamped to 0.8 .. 1.25 of the mean), so that all SMs
 //    finish together.  The speeds live in the workspace beside the arrival counters; a fresh workspace gives equal
