@@ -334,18 +334,24 @@ def run_ours(args, plan):
     mid = median_region(sampled)
     regions = plain + sampled
 
-    # ---- end to end: the step's inputs start in pinned host memory, the result ends there
-    # q, k_new and v_new of a step travel as ONE pinned host buffer and one copy (the caller's side of the API:
-    # the entry points take three pointers, which may point into one allocation)
-    parts = (q, k_new, v_new)
-    sizes = [t.numel() for t in parts]
-    hin = torch.cat([t.reshape(-1).cpu() for t in parts]).pin_memory()
-    din = torch.empty(sum(sizes), dtype=q.dtype, device=dev)
-    dq, dk, dv = (din[sum(sizes[:k]):sum(sizes[:k + 1])].view(parts[k].shape) for k in range(3))
+    # ---- end to end: the step's inputs start in pinned host memory, the result ends there.  One call of the
+    # library per step (puzzle_decode_step_host: three host-to-device copies, append, attention, one copy back),
+    # and the caller synchronises the stream before the next step because it reads the result on the host.  The
+    # context-sharded layer has no such entry point; there the copies are the caller's.
+    hin = torch.cat([t.reshape(-1).cpu() for t in (q, k_new, v_new)]).pin_memory()     # one buffer: one copy
+    hq = hin[: q.numel()].view(q.shape)
+    hk = hin[q.numel(): q.numel() + k_new.numel()].view(k_new.shape)
+    hv = hin[q.numel() + k_new.numel():].view(v_new.shape)
     hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    staging = torch.empty(P.puzzle_decode_step_host_staging_bytes(desc, w.batch), dtype=torch.uint8, device=dev)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new)
 
     def step_e2e(i):
-        din.copy_(hin, non_blocking=True)
+        if ctx is None and args.kernel == "mma":
+            P.puzzle_decode_step_host(desc, views[i % len(views)], hq, hk, hv, sinks, hout, staging, ws,
+                                      num_splits=args.splits, dev_status=status, stream=stream)
+            return
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
         P.puzzle_kv_append(desc, views_append[i % len(views)], dk, dv, dev_status=status, stream=stream)
         attention(i, dq)
         hout.copy_(out, non_blocking=True)

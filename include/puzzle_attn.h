@@ -231,6 +231,28 @@ PUZZLE_API puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* des
                                  int32_t num_splits, void* workspace, size_t workspace_bytes,
                                  int32_t* dev_status, void* stream);
 
+/* One whole layer-step for a caller whose step inputs and result live in HOST memory: copies q, k_new and v_new to
+ * the device, runs puzzle_kv_append and puzzle_decode_attn (the path of the paper's decode scenarios, Section
+ * "Optimized Scenarios", with the FP8 append of Section "KV Quantization"), and copies the bf16 result back, all
+ * enqueued on `stream`; the call returns without synchronising, so out_host is valid after the caller has
+ * synchronised the stream.  The cache, block table, lengths, scales and sinks stay on the device as for the
+ * other entry points.
+ *   q_host: host bf16 [batch][num_q_heads][head_dim];  k_new_host, v_new_host: host bf16 [batch][num_kv_heads][head_dim];
+ *   out_host: host bf16 [batch][num_q_heads][head_dim].  Pinned (page-locked) host memory keeps the copies
+ *     asynchronous; pageable memory works but serialises with the host.  When k_new_host follows q_host and
+ *     v_new_host follows k_new_host directly in memory (and the sizes are multiples of 256 bytes) the three travel
+ *     as one copy;
+ *   staging: device scratch of at least puzzle_decode_step_host_staging_bytes(desc, batch) bytes, 256-byte
+ *     aligned, owned by the caller (the library allocates nothing); not to be shared by steps that overlap;
+ *   num_splits, workspace, dev_status: as puzzle_decode_attn.
+ * Host-visible errors are reported before the first copy is enqueued. */
+PUZZLE_API size_t puzzle_decode_step_host_staging_bytes(const puzzle_layer_desc* desc, int32_t batch);
+PUZZLE_API puzzle_status puzzle_decode_step_host(const puzzle_layer_desc* desc, const puzzle_kv_view* kv,
+                                                 const void* q_host, const void* k_new_host, const void* v_new_host,
+                                                 const float* sinks, void* out_host, int32_t batch, int32_t num_splits,
+                                                 void* staging, size_t staging_bytes, void* workspace,
+                                                 size_t workspace_bytes, int32_t* dev_status, void* stream);
+
 /* Decode attention for up to n_q new tokens per sequence in one call: the tokens of a multi-token decode step, or
  * a chunk of a prompt after its bulk append (puzzle_kv_append_tokens), i.e. the input half of the paper's
  * fixed-length scenarios (Section "Optimized Scenarios"), on full and window layers (Section "Window attention for

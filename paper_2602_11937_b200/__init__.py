@@ -31,6 +31,8 @@ from .binding import (  # noqa: F401
     puzzle_decode_attn_tokens_workspace_bytes,
     puzzle_decode_attn_tokens_workspace_init,
     puzzle_decode_attn_workspace_bytes,
+    puzzle_decode_step_host,
+    puzzle_decode_step_host_staging_bytes,
     puzzle_decode_attn_workspace_init,
     puzzle_hbm_read_probe,
     puzzle_kv_amax_update,

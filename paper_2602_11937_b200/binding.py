@@ -30,6 +30,8 @@ EXPORTS = (
     "puzzle_decode_attn_tcgen05",
     "puzzle_decode_attn_static",
     "puzzle_decode_attn_partial",
+    "puzzle_decode_step_host",
+    "puzzle_decode_step_host_staging_bytes",
     "puzzle_decode_attn_tokens",
     "puzzle_decode_attn_tokens_workspace_bytes",
     "puzzle_decode_attn_tokens_workspace_init",
@@ -99,6 +101,11 @@ def _load():
         lib.puzzle_decode_attn_static.restype = ctypes.c_int
         lib.puzzle_decode_attn_static.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp,
                                                   i32, i32, vp, vp]
+        lib.puzzle_decode_step_host_staging_bytes.restype = sz
+        lib.puzzle_decode_step_host_staging_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32]
+        lib.puzzle_decode_step_host.restype = ctypes.c_int
+        lib.puzzle_decode_step_host.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(KVView), vp, vp, vp, vp, vp,
+                                                i32, i32, vp, sz, vp, sz, vp, vp]
         lib.puzzle_decode_attn_tokens_workspace_bytes.restype = sz
         lib.puzzle_decode_attn_tokens_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), i32, i32]
         lib.puzzle_decode_attn_tokens_workspace_init.restype = ctypes.c_int
@@ -297,6 +304,31 @@ def puzzle_decode_attn_static(desc: LayerDesc, view: KVView, q: torch.Tensor, si
                                              _p(lse_out, torch.float32, "lse_out"), q.shape[0], int(num_splits),
                                              _p(dev_status, torch.int32), _stream(stream)),
            "puzzle_decode_attn_static")
+
+
+def puzzle_decode_step_host_staging_bytes(desc: LayerDesc, batch: int) -> int:
+    return int(_load().puzzle_decode_step_host_staging_bytes(ctypes.byref(desc), int(batch)))
+
+
+def _host_ptr(t: torch.Tensor, name: str):
+    if t.is_cuda or not t.is_contiguous() or t.dtype != torch.bfloat16:
+        raise ValueError("%s must be a contiguous bf16 host tensor" % name)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def puzzle_decode_step_host(desc: LayerDesc, view: KVView, q_host: torch.Tensor, k_new_host: torch.Tensor,
+                            v_new_host: torch.Tensor, sinks: Optional[torch.Tensor], out_host: torch.Tensor,
+                            staging: torch.Tensor, workspace: torch.Tensor, num_splits: int = 0,
+                            dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Append + attention of one layer with q, k_new, v_new and out in host memory (pinned for asynchronous copies);
+    staging and workspace are device tensors.  Synchronise the stream before reading out_host."""
+    _check(_load().puzzle_decode_step_host(ctypes.byref(desc), ctypes.byref(view), _host_ptr(q_host, "q_host"),
+                                           _host_ptr(k_new_host, "k_new_host"), _host_ptr(v_new_host, "v_new_host"),
+                                           _p(sinks, torch.float32, "sinks"), _host_ptr(out_host, "out_host"),
+                                           q_host.shape[0], int(num_splits), _p(staging),
+                                           staging.numel() * staging.element_size(), _p(workspace),
+                                           workspace.numel() * workspace.element_size(), _p(dev_status, torch.int32),
+                                           _stream(stream)), "puzzle_decode_step_host")
 
 
 def puzzle_decode_attn_partial(desc: LayerDesc, view: KVView, q: torch.Tensor, o_part: torch.Tensor,

@@ -291,6 +291,57 @@ puzzle_status puzzle_decode_attn_tcgen05(const puzzle_layer_desc* desc, const pu
                           stream, true);
 }
 
+// Device staging of one step whose inputs and result live in host memory: q, k_new, v_new, out, each padded to 256 bytes.
+static size_t staging_part(size_t elems) { return (elems * sizeof(__nv_bfloat16) + 255) & ~(size_t)255; }
+
+size_t puzzle_decode_step_host_staging_bytes(const puzzle_layer_desc* desc, int32_t batch) {
+  if (check_desc(desc) != PUZZLE_OK || batch <= 0 || batch > kMaxBatch) return 0;
+  const size_t qn = (size_t)batch * desc->num_q_heads * desc->head_dim, kn = (size_t)batch * desc->num_kv_heads * desc->head_dim;
+  return 2 * staging_part(qn) + 2 * staging_part(kn);
+}
+
+puzzle_status puzzle_decode_step_host(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q_host,
+                                      const void* k_new_host, const void* v_new_host, const float* sinks,
+                                      void* out_host, int32_t batch, int32_t num_splits, void* staging,
+                                      size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                      int32_t* dev_status, void* stream) {
+  if (!q_host || !k_new_host || !v_new_host || !out_host) return PUZZLE_ERR_NULL;
+  const size_t need = puzzle_decode_step_host_staging_bytes(desc, batch);
+  if (need == 0) return check_desc(desc) != PUZZLE_OK ? check_desc(desc) : PUZZLE_ERR_SHAPE;
+  if (!staging || staging_bytes < need || (reinterpret_cast<uintptr_t>(staging) & 255)) return PUZZLE_ERR_WORKSPACE;
+  const size_t qn = (size_t)batch * desc->num_q_heads * desc->head_dim, kn = (size_t)batch * desc->num_kv_heads * desc->head_dim;
+  char* dq = static_cast<char*>(staging);
+  char* dk = dq + staging_part(qn);
+  char* dv = dk + staging_part(kn);
+  char* dout = dv + staging_part(kn);
+  // every host-visible error of the two device calls is found before the first copy is enqueued
+  puzzle_status st = check_decode_attn_args(desc, kv, dq, dout, batch, num_splits, false);
+  if (st != PUZZLE_OK) return st;
+  if (!workspace || workspace_bytes < puzzle_decode_attn_workspace_bytes(desc, batch, num_splits) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 15))
+    return PUZZLE_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t qb = qn * sizeof(__nv_bfloat16), kb = kn * sizeof(__nv_bfloat16);
+  const char* hq = static_cast<const char*>(q_host);
+  if (static_cast<const char*>(k_new_host) == hq + qb && static_cast<const char*>(v_new_host) == hq + qb + kb &&
+      qb % 256 == 0 && kb % 256 == 0) {
+    // the three inputs follow each other in host memory as they do in the staging area: one copy
+    if (cudaMemcpyAsync(dq, q_host, qb + 2 * kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return PUZZLE_ERR_CUDA;
+  } else if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+             cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+             cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+    return PUZZLE_ERR_CUDA;
+  }
+  st = puzzle_kv_append(desc, kv, dk, dv, batch, dev_status, stream);
+  if (st != PUZZLE_OK) return st;
+  st = puzzle_decode_attn(desc, kv, dq, sinks, dout, nullptr, batch, num_splits, workspace, workspace_bytes, dev_status,
+                          stream);
+  if (st != PUZZLE_OK) return st;
+  return cudaMemcpyAsync(out_host, dout, qn * sizeof(__nv_bfloat16), cudaMemcpyDeviceToHost, s) == cudaSuccess
+             ? PUZZLE_OK
+             : PUZZLE_ERR_CUDA;
+}
+
 puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* q,
                                          float* o_part, float* lse_part, int32_t batch, int32_t num_splits,
                                          void* workspace, size_t workspace_bytes, int32_t* dev_status,

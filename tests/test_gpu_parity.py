@@ -307,3 +307,33 @@ def test_host_side_argument_errors():
         P.puzzle_kv_append(dev.desc(), v, dev.k_new, dev.v_new)
     assert e.value.code == 1
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------ host-buffer layer-step --
+
+def test_step_with_host_buffers_matches_the_device_path_and_the_oracle():
+    """puzzle_decode_step_host: q, k_new, v_new in pinned host memory, result in pinned host memory; the cache gets
+    the oracle's bytes and the output the oracle's values."""
+    import paper_2602_11937_b200 as P
+    from gpu_helpers import assert_close
+    w = synth.workload(2, scale=0.1)
+    case = make_case(w)
+    dev = _dev(case)
+    d = dev.desc(0)
+    hq, hk, hv = (t.cpu().pin_memory() for t in (dev.q, dev.k_new, dev.v_new))
+    hout = torch.zeros(w.batch, w.hq, w.head_dim, dtype=torch.bfloat16).pin_memory()
+    staging = torch.empty(P.puzzle_decode_step_host_staging_bytes(d, w.batch), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(d, w.batch, 0), dtype=torch.uint8, device="cuda")
+    P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
+    P.puzzle_decode_step_host(d, dev.view(), hq, hk, hv, dev.sinks, hout, staging, ws, dev_status=dev.status)
+    torch.cuda.synchronize()
+    oracle_append(case)
+    gk, gv = dev.cache_bytes()
+    assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
+    ref, _ = oracle_attn(case, 0)
+    assert_close(hout.float().numpy().astype(np.float64), ref, "host-buffer step")
+    assert int(dev.status.item()) == 0
+    with pytest.raises(P.PuzzleError) as e:          # staging too small: nothing is enqueued
+        P.puzzle_decode_step_host(d, dev.view(), hq, hk, hv, dev.sinks, hout, staging[:256], ws)
+    assert e.value.code == 4
+    torch.cuda.synchronize()
