@@ -155,10 +155,15 @@ PUZZLE_API puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, 
  * context length (the grid is persistent), so there is no max_seq_len argument. */
 PUZZLE_API size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits);
 
-/* Prepares a freshly allocated workspace: zero-fills the arrival counters and
- * the CTA-speed words at its start (padded to 256 bytes) on `stream`.  Call it once per workspace before its first puzzle_decode_attn;
- * every completed puzzle_decode_attn leaves the counters at zero again, for any
- * batch and split choice that fits the workspace.  Call it again after a step
+/* Prepares a freshly allocated workspace: zero-fills the CTA-speed words and
+ * the arrival counters at its start on `stream`.  Call it once per workspace
+ * before its first puzzle_decode_attn; every completed puzzle_decode_attn
+ * leaves the counters at zero again.  The counter block has room for 16384
+ * (sequence, KV head) pairs whatever `batch` is, and the partials start behind
+ * it: a workspace prepared once serves calls of any batch with
+ * batch * num_kv_heads <= 16384 and any split choice that fit it, one after
+ * the other.  (A larger batch moves the partials: prepare the workspace for
+ * that batch and use it for that batch only.)  Call it again after a step
  * whose *dev_status reported PUZZLE_DEV_WAIT_EXPIRED (that step stopped half
  * way).  The split-KV phase of Section "Optimized Scenarios"' KV-bound decode
  * needs these counters to know which worker finishes a (sequence, KV head). */

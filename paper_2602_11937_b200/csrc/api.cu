@@ -97,10 +97,16 @@ int grid_ctas() { return device_info().sm_count > 0 ? device_info().sm_count : 1
 
 int decode_warps(int kv_dtype) { return kv_dtype == PUZZLE_KV_FP8_E4M3 ? kDecodeWarpsFp8 : kDecodeWarpsBf16; }
 
-// The workspace starts with one arrival counter per (sequence, KV head) and the CTA-speed words of the CTA-balanced
-// kernel, padded to 256 bytes.
+// The workspace starts with the CTA-speed words of the CTA-balanced kernel, then one arrival counter per (sequence,
+// KV head), then the partials.  Every completed call leaves the arrival counters at zero.  The counter block has room
+// for kCounterFloor counters whatever the batch, so that up to that many (sequence, KV head) pairs the partials of
+// one call never lie where another call's counters do: one prepared workspace then serves calls of different batch
+// sizes one after the other.  Beyond the floor the layout follows the batch.
+constexpr size_t kCounterFloor = 16384;
+size_t cta_word_bytes() { return (cta_rate_words(grid_ctas()) * sizeof(int32_t) + 255) & ~(size_t)255; }
 size_t counter_bytes(int batch, int Hkv) {
-  return (((size_t)batch * Hkv + cta_rate_words(grid_ctas())) * sizeof(int32_t) + 255) & ~(size_t)255;
+  const size_t n = std::max((size_t)batch * Hkv, kCounterFloor);
+  return cta_word_bytes() + ((n * sizeof(int32_t) + 255) & ~(size_t)255);
 }
 
 // The balanced schedule runs on the CTA-balanced kernel when the batch fits its shared-memory schedule and the
@@ -246,7 +252,8 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   P.v_scale = kv->v_scale;
   P.part_o = part_o;
   P.part_lse = part_lse;
-  P.counters = static_cast<int32_t*>(workspace);
+  P.cta_words = static_cast<int32_t*>(workspace);
+  P.counters = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + cta_word_bytes());
   P.sinks = sinks;
   P.out = out_f32 ? nullptr : static_cast<__nv_bfloat16*>(out);
   P.out_f32 = out_f32 ? static_cast<float*>(out) : nullptr;
@@ -351,8 +358,10 @@ puzzle_status puzzle_decode_attn_partial(const puzzle_layer_desc* desc, const pu
                           dev_status, stream, false, true);
 }
 
+// Room for the largest supported batch * ceil(n_q / 2) whatever the call's own, for the same reason as counter_bytes.
 static size_t tokens_counter_bytes(int batch, int n_q, int Hkv) {
-  return (decode_attn_tokens_counters(batch, n_q, Hkv) * sizeof(int32_t) + 255) & ~(size_t)255;
+  const size_t n = std::max<size_t>(decode_attn_tokens_counters(batch, n_q, Hkv), (size_t)kTokMaxRows * Hkv);
+  return (n * sizeof(int32_t) + 255) & ~(size_t)255;
 }
 
 size_t puzzle_decode_attn_tokens_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t n_q) {

@@ -21,6 +21,7 @@ struct alignas(64) DecodeParams {
   float* part_o;
   float* part_lse;
   int32_t* counters;   // [batch*Hkv] arrivals per (sequence, KV head); zero before and after every launch
+  int32_t* cta_words;  // CTA-balanced kernel only: its CTA counter, buffer switch and the two speed buffers
   const float* sinks;  // [Hq] or null
   __nv_bfloat16* out;  // [batch][Hq][D]
   float* out_f32;      // when set, the merged rows are stored here as float32 instead (out is unused)
@@ -53,7 +54,7 @@ constexpr int kDecodeWarpsFp8 = 12, kDecodeStagesFp8 = 2, kTileFp8 = 64;
 constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
 // The CTA-balanced kernel keeps its schedule arrays beside the TMA rings and the deposit buffers in shared memory,
 // which bounds the batch it takes.  Launches with at least kCtaRateMinTiles tiles per CTA note the speed of every
-// CTA slot in the workspace (after the arrival counters: a CTA counter, the buffer switch, two pad words, then two
+// CTA slot at the start of the workspace (before the arrival counters: a CTA counter, the buffer switch, two pad words, then two
 // float buffers of one speed per CTA) and are cut by the speeds the launch before them noted.
 constexpr int kCtaMaxBatch = 1024;
 constexpr int kCtaMinTilesPerCta = 64;   // below this bound on the tiles per CTA the warp-scheduled kernel is used

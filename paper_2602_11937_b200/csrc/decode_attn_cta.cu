@@ -14,8 +14,8 @@
 //    together.  (Only the very first chunk of every warp is fixed at set-up, when all twelve lie in one pair.)
 //  * On large launches every CTA notes how many tiles per cycle it managed; the next large launch on the same
 //    workspace cuts the ranges in proportion to those speeds (clamped to 0.8 .. 1.25 of the mean), so that all SMs
-//    finish together.  The speeds live in the workspace beside the arrival counters; a fresh workspace gives equal
-//    ranges.  They change how the work is cut, never what is computed.
+//    finish together.  The speeds live at the start of the workspace, before the arrival counters; a fresh
+//    workspace gives equal ranges.  They change how the work is cut, never what is computed.
 //
 // A "piece" is the part of one pair inside one CTA's range.  A warp that leaves a piece deposits its running
 // (max, sum, accumulator) in a shared-memory buffer of its own and adds its tile count to the piece's counter; the
@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
   int* cum = reinterpret_cast<int*>(sp);
 
   // speeds of the CTA slots from earlier launches: two buffers, the valid one named by `epoch`
-  int* cta_done = P.counters + P.batch * P.Hkv;
+  int* cta_done = P.cta_words;
   int* epoch_p = cta_done + 1;
   float* rates = reinterpret_cast<float*>(cta_done + 4);
 

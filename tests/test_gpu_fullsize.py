@@ -139,7 +139,7 @@ def test_cta_speeds_change_the_cut_not_the_result():
     ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
     P.puzzle_decode_attn_workspace_init(d, w.batch, ws)
     words = ws.view(torch.int32)
-    first = w.batch * w.hkv + 4               # after the arrival counters, the CTA counter, the switch and two pad words
+    first = 4                                 # the workspace starts with the CTA counter, the switch and two pad words
     n_sm = torch.cuda.get_device_properties(0).multi_processor_count
     rng = np.random.default_rng(5)
     hk, hv = case.host
@@ -166,7 +166,9 @@ def test_cta_speeds_change_the_cut_not_the_result():
             assert np.isfinite(got_all).all()
             got = np.stack([got_all[b, h] for b, h in items])
             assert_close(got, ref, "speed words: %s" % ("zero" if fill is None else "filled"))
-    assert not words[: w.batch * w.hkv + 1].any()      # arrival counters and the CTA counter are back at zero
+    n_cta_words = ((4 + 2 * n_sm) * 4 + 255) // 256 * 64       # the CTA words are padded to 256 bytes
+    assert int(words[0]) == 0                           # the CTA counter is back at zero ...
+    assert not words[n_cta_words: n_cta_words + 16384].any()   # ... and so is the whole block of arrival counters
 
 
 def test_full_size_ragged_stack_layers():

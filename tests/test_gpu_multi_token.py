@@ -95,6 +95,21 @@ def test_tokens_kernel_shares_tiles_between_query_tokens(window, n_q):
     """puzzle_decode_attn_tokens (pairs of query tokens on one pass over the tiles) against the oracle's
     single-token step at every query position: ragged numbers of new tokens, sequences shorter than a tile, one
     with no query, contexts that span many workers."""
+    _tokens_against_oracle(window, n_q, None)
+
+
+def test_tokens_kernel_one_workspace_for_different_token_counts():
+    """One workspace, prepared once, serves calls with different numbers of query tokens one after the other."""
+    import paper_2602_11937_b200 as P
+    d = P.layer_desc(kv_dtype=P.KV_FP8_E4M3)
+    ws = torch.empty(P.puzzle_decode_attn_tokens_workspace_bytes(d, 6, 5), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    P.puzzle_decode_attn_tokens_workspace_init(d, 6, 1, ws)
+    for n_q in (5, 2, 4, 1, 5):
+        _tokens_against_oracle(0, n_q, ws)
+
+
+def _tokens_against_oracle(window, n_q, shared_ws):
     import paper_2602_11937_b200 as P
     from gpu_helpers import DeviceCase, assert_close
     w = synth.Workload("tokq", 1, 6, 3000, [0], paged=True)
@@ -107,9 +122,11 @@ def test_tokens_kernel_shares_tiles_between_query_tokens(window, n_q):
     d = dev.desc(window)
     P.puzzle_kv_append_tokens(d, dev.view(), k.cuda(), v.cuda(), ql_dev, dev_status=dev.status)
     _oracle_append_chunk(case, lens_after, q_lens, k, v)
-    ws = torch.empty(P.puzzle_decode_attn_tokens_workspace_bytes(d, w.batch, n_q), dtype=torch.uint8, device="cuda")
-    ws.fill_(0xFF)
-    P.puzzle_decode_attn_tokens_workspace_init(d, w.batch, n_q, ws)
+    ws = shared_ws
+    if ws is None:
+        ws = torch.empty(P.puzzle_decode_attn_tokens_workspace_bytes(d, w.batch, n_q), dtype=torch.uint8, device="cuda")
+        ws.fill_(0xFF)
+        P.puzzle_decode_attn_tokens_workspace_init(d, w.batch, n_q, ws)
     for call in range(2):          # the second call finds the counters as the first one left them
         out = torch.full((w.batch, n_q, w.hq, w.head_dim), 7.0, dtype=torch.bfloat16, device="cuda")
         lse = torch.full((w.batch, n_q, w.hq), 7.0, dtype=torch.float32, device="cuda")

@@ -269,7 +269,7 @@ def test_split_partials_are_what_the_oracle_computes_per_split():
     head = nbytes - rows * 65 * 4              # the partials follow the block of counters (a multiple of 256 bytes)
     assert head > 0 and head % 256 == 0
     part = ws[head // 4:]
-    assert not ws[:1].any()                    # the pair's arrival counter: a finished call leaves it at zero
+    assert not ws[(head - 16384 * 4) // 4: head // 4].any()   # the block of arrival counters (it ends where the partials start): a finished call leaves it at zero
     po = part[: rows * 64].reshape(64, 2, 64).cpu().numpy().astype(np.float64)
     pl = part[rows * 64: rows * 65].reshape(64, 2).cpu().numpy().astype(np.float64)
     for s, (t0, t1) in enumerate([(0, 128), (128, 256)]):
@@ -337,3 +337,31 @@ def test_step_with_host_buffers_matches_the_device_path_and_the_oracle():
         P.puzzle_decode_step_host(d, dev.view(), hq, hk, hv, dev.sinks, hout, staging[:256], ws)
     assert e.value.code == 4
     torch.cuda.synchronize()
+
+
+def test_one_workspace_serves_calls_of_different_batch_sizes():
+    """A workspace sized for the largest batch is prepared once and then used by calls of different batch sizes,
+    schedules and kernels one after the other: every completed call leaves the counters at zero, and neither the
+    counters nor what the CTA-balanced kernel keeps between calls sit where another batch size puts its partials."""
+    import paper_2602_11937_b200 as P
+    from gpu_helpers import assert_close
+    cases = []
+    for batch, ctx in ((3, 500), (9, 300), (1, 900), (6, 200)):
+        w = synth.Workload("ws%d" % batch, batch, batch, ctx, [0], paged=True)
+        case = make_case(w)
+        dev = _dev(case)
+        dev.append(); oracle_append(case)
+        cases.append((w, dev, oracle_attn(case, 0)[0]))
+    d = cases[0][1].desc(0)
+    ws = torch.empty(max(P.puzzle_decode_attn_workspace_bytes(d, 9, s) for s in (0, 5)), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    P.puzzle_decode_attn_workspace_init(d, 3, ws)          # prepared for one batch size, used with others
+    for rnd in range(2):
+        for w, dev, ref in cases:
+            for sched in (P.SCHED_CTA, P.SCHED_WARP, 5, P.SCHED_AUTO):
+                out = torch.full((w.batch, w.hq, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+                P.puzzle_decode_attn(d, dev.view(), dev.q, dev.sinks, out, None, num_splits=sched, workspace=ws,
+                                     dev_status=dev.status)
+                torch.cuda.synchronize()
+                assert int(dev.status.item()) == 0
+                assert_close(out.float().cpu().numpy().astype(np.float64), ref, "batch %d sched %d" % (w.batch, sched))

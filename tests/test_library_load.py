@@ -37,8 +37,10 @@ def test_status_strings_and_workspace_size_need_no_gpu():
     a = P.puzzle_decode_attn_workspace_bytes(d, 16, 0)
     b = P.puzzle_decode_attn_workspace_bytes(d, 16, 8)
     partials = 16 * 64 * 8 * 65 * 4                     # 8 splits of (o, lse) per (sequence, query head)
-    head = b - partials                                 # arrival counters + CTA-speed words (these grow with the SM count)
-    assert a > 0 and head % 256 == 0 and head >= (16 * 8 + 4 + 2) * 4
+    head = b - partials                                 # CTA-speed words (these grow with the SM count) + arrival counters
+    assert a > 0 and head % 256 == 0 and head >= 256 + 16384 * 4
+    big = P.puzzle_decode_attn_workspace_bytes(d, 4096, 1) - 4096 * 64 * 65 * 4
+    assert big - head == (4096 * 8 - 16384) * 4         # the counter block grows with the batch only beyond its floor
     bad = P.layer_desc(head_dim=128)
     assert P.puzzle_decode_attn_workspace_bytes(bad, 16, 0) == 0
 
