@@ -23,7 +23,11 @@
  *     shared-memory limit it has set on its kernels, the address of the
  *     built-in scratch array).  Work is enqueued on the CUDA stream passed as
  *     `stream` (a cudaStream_t cast to void*; NULL is the default stream) and
- *     the call returns without synchronising.
+ *     the call returns without synchronising.  Stream order holds as usual: a
+ *     kernel of the library reads or writes global memory only after all
+ *     earlier work on its stream has completed (some are launched so that
+ *     their thread blocks are placed, and set up shared memory, while the
+ *     kernel before them drains; nothing else runs early).
  *   - The balanced schedule hands tiles of the cache to warps as they become
  *     free, so the order of the float32 sums can differ between two calls on the
  *     same inputs: outputs agree to rounding (the last bit of a bf16 value may

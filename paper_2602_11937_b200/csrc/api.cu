@@ -180,12 +180,13 @@ puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_vi
   if (!k_new || !v_new) return PUZZLE_ERR_NULL;
   const long long threads = 2ll * batch * desc->num_kv_heads * (kHeadDim / 2);
   const int grid = (int)((threads + 255) / 256);
-  kv_append_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      kv->k_cache, kv->v_cache, static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
-      kv->block_table, kv->seq_lens, kv->k_scale, kv->v_scale, kv->num_blocks, batch, desc->num_kv_heads,
-      kv->max_blocks_per_seq, desc->kv_dtype, dev_status);
+  const cudaError_t e = launch_dependent(
+      kv_append_kernel, dim3(grid), dim3(256), 0, static_cast<cudaStream_t>(stream), kv->k_cache, kv->v_cache,
+      static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), kv->block_table,
+      kv->seq_lens, kv->k_scale, kv->v_scale, kv->num_blocks, batch, desc->num_kv_heads, kv->max_blocks_per_seq,
+      desc->kv_dtype, dev_status);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+  return e == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
 }
 
 puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* k_new,

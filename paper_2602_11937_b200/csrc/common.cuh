@@ -19,6 +19,34 @@ constexpr int kMaxBatch = 4096;
 
 void count_launch();
 
+// --------------------------------------------- programmatic dependent launch --
+// The append and the two balanced decode kernels are launched so that their CTAs may be placed on an SM as soon as
+// the kernel before them on the stream lets go of it, instead of after that whole grid has drained and a launch
+// latency on top.  A kernel launched this way calls grid_dependency_wait() before its first access to global memory:
+// it returns once every earlier kernel on the stream has completed and its writes are visible, so nothing the caller
+// (or an earlier call) produced is read early; all that runs ahead of it is the placement of the CTA and set-up that
+// touches shared memory and kernel parameters only.  release_dependents() at the top of a decode kernel tells the
+// kernel behind it (if it was launched this way) that its CTAs may be placed whenever there is room; a kernel that
+// never calls it releases them when its last CTA exits.  Both are no-ops next to a kernel launched the ordinary way.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

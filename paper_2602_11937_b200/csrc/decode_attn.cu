@@ -133,6 +133,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     tma_prefetch_desc(&P.tmK);
     tma_prefetch_desc(&P.tmV);
   }
+  release_dependents();
+  grid_dependency_wait();   // nothing above reads or writes global memory
   build_schedule(cum, lens, P.seq_lens, P.batch, P.Hkv, P.window, P.max_blocks_per_seq * kBlock, TT, P.dev_status);
 
   const int nW = gridDim.x * NW;
@@ -251,8 +253,7 @@ static cudaError_t launch_variant(const DecodeParams& P, int ctas, cudaStream_t 
   }
   const size_t need = smem_bytes_of<NW, NS, TT, FP8>(P.batch);
   if (need > (size_t)smem_limit) return cudaErrorInvalidValue;  // batch too large for the schedule arrays
-  kern<<<ctas, NW * 32, need, s>>>(P);
-  return cudaGetLastError();
+  return launch_dependent(kern, dim3(ctas), dim3(NW * 32), need, s, P);
 }
 
 cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit) {

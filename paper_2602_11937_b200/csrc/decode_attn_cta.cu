@@ -50,7 +50,7 @@ constexpr int kPieceSlots = 16;  // tile counters of open pieces; pieces k and k
 // Hand-out state of a CTA (shared memory); the first 16 bytes are read by one load.
 struct alignas(16) CtaCtl {
   int pos, end, lo, p_first;  // next tile to hand out; the CTA's range [lo, end) of the tile space; its first pair
-  long long t0;               // clock at kernel entry
+  long long t0;               // clock when the kernels before this one had completed
   int warps_left;             // warps still running: the last one notes the CTA's speed
   int use_rates;              // this launch is large enough to note (and use) CTA speeds
   int4 seed[2];               // the pair the range starts in, as a PairCache record: every warp starts from it
@@ -296,10 +296,15 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
     fence_mbar_init();
   }
   if (threadIdx.x == 0) {
-    ctl.t0 = clock64();
     tma_prefetch_desc(&P.tmK);
     tma_prefetch_desc(&P.tmV);
   }
+  if (threadIdx.x < 32) dep_piece[threadIdx.x] = -1;
+  if (threadIdx.x < kPieceSlots) { pk_key[threadIdx.x] = -1; pk_done[threadIdx.x] = 0; }
+  if (threadIdx.x == 0) cum[0] = 0;
+  release_dependents();
+  grid_dependency_wait();   // nothing above reads or writes global memory
+  if (threadIdx.x == 0) ctl.t0 = clock64();
   // ---- schedule, step 1: tiles of every sequence
   for (int b = threadIdx.x; b < P.batch; b += blockDim.x) {
     bool too_long;
@@ -307,9 +312,6 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_cta_kernel(const __gri
     if (too_long && P.dev_status && blockIdx.x == 0) atomicOr(P.dev_status, (int)PUZZLE_DEV_SEQ_TOO_LONG);
     cum[b + 1] = r.ntile * P.Hkv;
   }
-  if (threadIdx.x < 32) dep_piece[threadIdx.x] = -1;
-  if (threadIdx.x < kPieceSlots) { pk_key[threadIdx.x] = -1; pk_done[threadIdx.x] = 0; }
-  if (threadIdx.x == 0) cum[0] = 0;
   // one warp turns the noted speeds into cumulative shares (fixed point, 4096 = the mean speed); without a full set
   // of speeds every CTA gets the same share
   if (warp == 1) {
@@ -694,8 +696,7 @@ static cudaError_t launch_cta_variant(const DecodeParams& P, int ctas, cudaStrea
   }
   const size_t need = cta_smem_bytes<NW, NS, TT, FP8>(P.batch, ctas);
   if (need > (size_t)smem_limit) return cudaErrorInvalidValue;
-  kern<<<ctas, NW * 32, need, s>>>(P);
-  return cudaGetLastError();
+  return launch_dependent(kern, dim3(ctas), dim3(NW * 32), need, s, P);
 }
 
 cudaError_t launch_decode_attn_cta(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit) {

@@ -21,6 +21,9 @@ __global__ void __launch_bounds__(256) kv_append_kernel(void* k_cache, void* v_c
                                                         const float* v_scale, long long num_blocks, int batch,
                                                         int Hkv, int max_blocks_per_seq, int kv_dtype,
                                                         int32_t* dev_status) {
+  // No early release here: the decode kernel behind the append should find every SM free when its CTAs are placed, so
+  // that CTA i lands on the same SM launch after launch (the CTA speeds it notes are speeds of SMs).
+  grid_dependency_wait();
   const int pairs_per_tensor = batch * Hkv * (kHeadDim / 2);
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= 2 * pairs_per_tensor) return;

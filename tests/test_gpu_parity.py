@@ -365,3 +365,59 @@ def test_one_workspace_serves_calls_of_different_batch_sizes():
                 torch.cuda.synchronize()
                 assert int(dev.status.item()) == 0
                 assert_close(out.float().cpu().numpy().astype(np.float64), ref, "batch %d sched %d" % (w.batch, sched))
+
+
+@pytest.mark.parametrize("sched", ["auto", "cta"])
+def test_stream_order_holds_next_to_kernels_of_the_caller(sched):
+    """Decode steps enqueued back to back with no host synchronisation, the caller's own kernels in between: one that
+    advances the sequence lengths on the device, others that produce this step's q, k_new and v_new right before the
+    library reads them, one that consumes the output right after.  The library's kernels are placed early (their
+    thread blocks may sit on an SM while the kernel before them drains) but must not read any of this early: every
+    step's output and the final cache bytes are checked against the oracle."""
+    import paper_2602_11937_b200 as P
+    from gpu_helpers import assert_close
+    steps, batch, ctx = 40, 4, 700
+    w = synth.Workload("order", 1, batch, ctx, [0], paged=True)
+    start = np.array([ctx - steps, 0, 37, 300], dtype=np.int32)
+    case = make_case(w, seq_lens=start + 1)               # the helpers fill the cache below the first appended token
+    dev = _dev(case)
+    d = dev.desc(0)
+    num = P.SCHED_CTA if sched == "cta" else P.SCHED_AUTO
+    ws = torch.zeros(P.puzzle_decode_attn_workspace_bytes(d, batch, num), dtype=torch.uint8, device="cuda")
+    P.puzzle_decode_attn_workspace_init(d, batch, ws)
+    g = torch.Generator().manual_seed(77)
+    qs = torch.randn(steps, batch, w.hq, w.head_dim, generator=g).to(torch.bfloat16)
+    ks = torch.randn(steps, batch, w.hkv, w.head_dim, generator=g).to(torch.bfloat16)
+    vs = torch.randn(steps, batch, w.hkv, w.head_dim, generator=g).to(torch.bfloat16)
+    qs_d, ks_d, vs_d = qs.cuda(), ks.cuda(), vs.cuda()
+    lens_dev = torch.from_numpy(start).cuda()
+    view = P.kv_view(dev.k_cache, dev.v_cache, lens_dev, block_table=dev.table, max_blocks_per_seq=w.blocks_per_seq,
+                     k_scale=dev.k_scale, v_scale=dev.v_scale)
+    q = torch.zeros(batch, w.hq, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    k_new = torch.zeros(batch, w.hkv, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    v_new = torch.zeros_like(k_new)
+    out = torch.zeros_like(q)
+    kept = torch.zeros(steps, batch, w.hq, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    torch.cuda.synchronize()
+    for t in range(steps):                                 # nothing in this loop waits for the GPU
+        lens_dev.add_(1)
+        torch.mul(ks_d[t], 1, out=k_new)
+        torch.mul(vs_d[t], 1, out=v_new)
+        P.puzzle_kv_append(d, view, k_new, v_new, dev_status=dev.status)
+        torch.mul(qs_d[t], 1, out=q)
+        P.puzzle_decode_attn(d, view, q, dev.sinks, out, None, num_splits=num, workspace=ws, dev_status=dev.status)
+        torch.mul(out, 1, out=kept[t])
+    torch.cuda.synchronize()
+    assert int(dev.status.item()) == 0
+    got = kept.float().cpu().numpy().astype(np.float64)
+    for t in range(steps):
+        lens = (start + t + 1).astype(np.int32)
+        oracle.kv_append(case["k_cache"], case["v_cache"], case["kv_dtype"], w.block, case["table"], w.blocks_per_seq,
+                         lens, case["k_scale"], case["v_scale"], bf16_bits(ks[t]), bf16_bits(vs[t]))
+        if t % 3 == 0 or t == steps - 1:
+            ref, _ = oracle.decode_attn(case["k_cache"], case["v_cache"], case["kv_dtype"], case["table"],
+                                        w.blocks_per_seq, lens, case["k_scale"], case["v_scale"], bf16_bits(qs[t]),
+                                        case["sinks"], 0, case["sm_scale"])
+            assert_close(got[t], ref.reshape(got[t].shape), "step %d" % t)
+    gk, gv = dev.cache_bytes()
+    assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
