@@ -113,13 +113,18 @@ size_t counter_bytes(int batch, int Hkv) {
 // launch can be large: with at most a few tiles per warp (window layers, short contexts) a launch is a chain of
 // latencies, which the warp-scheduled kernel's shorter set-up serves better.  The bound on the tiles comes from
 // what the host knows: the window, or the length of a block-table row.
-bool use_cta_kernel(const puzzle_layer_desc* d, const puzzle_kv_view* kv, int batch, int num_splits) {
-  if (num_splits == PUZZLE_SCHED_CTA) return true;
-  if (num_splits != 0 || batch > kCtaMaxBatch) return false;
+// Upper bound on the tiles of one (sequence, KV head) from what the host knows.
+long long tiles_per_pair_bound(const puzzle_layer_desc* d, const puzzle_kv_view* kv) {
   const int tt = d->kv_dtype == PUZZLE_KV_FP8_E4M3 ? kTileFp8 : kTileBf16;
   long long per_pair = ((long long)kv->max_blocks_per_seq * kBlock + tt - 1) / tt;
   if (d->window > 0) per_pair = std::min<long long>(per_pair, (d->window + tt - 1) / tt + 1);
-  return per_pair * batch * d->num_kv_heads >= (long long)kCtaMinTilesPerCta * grid_ctas();
+  return per_pair;
+}
+
+bool use_cta_kernel(const puzzle_layer_desc* d, const puzzle_kv_view* kv, int batch, int num_splits) {
+  if (num_splits == PUZZLE_SCHED_CTA) return true;
+  if (num_splits != 0 || batch > kCtaMaxBatch) return false;
+  return tiles_per_pair_bound(d, kv) * batch * d->num_kv_heads >= (long long)kCtaMinTilesPerCta * grid_ctas();
 }
 
 size_t workspace_floats(int batch, int Hkv, int num_splits, int kv_dtype) {
@@ -276,6 +281,10 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   } else if (use_cta_kernel(desc, kv, batch, num_splits)) {
     le = launch_decode_attn_cta(P, fp8, ctas, s, device_info().smem_limit + 3);
   } else {
+    // Narrow windows and short contexts: with at most kWholePairTiles tiles per (sequence, KV head) a pair is not cut
+    // at all.  One warp takes it whole and stores the output itself, which drops the partial, the arrival and the
+    // merge (three dependent trips through L2) from a launch that is a chain of latencies anyway.
+    if (splits == 0 && tiles_per_pair_bound(desc, kv) <= kWholePairTiles) P.num_splits = 1;
     le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
   }
   if (le != cudaSuccess) return PUZZLE_ERR_CUDA;

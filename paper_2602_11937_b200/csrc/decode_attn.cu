@@ -147,7 +147,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     cc.end = min(cc.pos + q, T);
     cc.step = 0;
   } else {
-    cc.pos = w;
+    // consecutive units go to different SMs: a launch with fewer units than workers still uses every SM
+    cc.pos = warp * gridDim.x + blockIdx.x;
     cc.end = P.batch * P.Hkv * P.num_splits;
     cc.step = nW;
   }
@@ -177,6 +178,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     st.template load_query<FP8>(P.q + ((size_t)cs.b * (P.Hkv * kGroup) + cs.kvh * kGroup + g) * kHeadDim,
                                 P.k_scale && FP8 ? P.k_scale[cs.kvh] : 1.f, P.sm_scale_log2e, c);
     st.reset();
+    // one split per pair: this warp's result is final, so the sink is fetched while the tiles are in flight
+    const float sink_g = (P.num_splits == 1 && P.sinks) ? P.sinks[cs.kvh * kGroup + g] : -INFINITY;
 
 #pragma unroll 1
     for (int t = cs.t; t < cs.t_end; ++t) {
@@ -206,6 +209,33 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
     l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
     const float vs = P.v_scale && FP8 ? P.v_scale[cs.kvh] : 1.f;
+    if (P.num_splits == 1) {
+      // the whole (sequence, KV head) was this warp's: fold the sink in and store the output, no partial, no arrival
+      const long long row_out = (long long)cs.b * (P.Hkv * kGroup) + cs.kvh * kGroup + g;
+      const float s2 = sink_g * 1.4426950408889634f;
+      const float M = fmaxf(l_tot > 0.f ? st.m_ref : -INFINITY, s2);
+      float f = 0.f, Z = 0.f;
+      if (M != -INFINITY) {
+        const float wa = l_tot > 0.f ? ex2(st.m_ref - M) : 0.f;
+        Z = l_tot * wa + (s2 == -INFINITY ? 0.f : ex2(s2 - M));
+        f = wa * vs / Z;
+      }
+      if (P.out_f32) {
+        float* dst = P.out_f32 + row_out * kHeadDim + 2 * c;
+#pragma unroll
+        for (int nd = 0; nd < 8; ++nd)
+          *reinterpret_cast<float2*>(dst + 8 * nd) =
+              make_float2((st.O[nd][0] + st.O[nd][2]) * f, (st.O[nd][1] + st.O[nd][3]) * f);
+      } else {
+        __nv_bfloat16* dst = P.out + row_out * kHeadDim + 2 * c;
+#pragma unroll
+        for (int nd = 0; nd < 8; ++nd)
+          *reinterpret_cast<uint32_t*>(dst + 8 * nd) =
+              f32x2_to_bf16x2((st.O[nd][0] + st.O[nd][2]) * f, (st.O[nd][1] + st.O[nd][3]) * f);
+      }
+      if (P.lse_out && c == 0) P.lse_out[row_out] = Z > 0.f ? (M + log2f(Z)) * 0.6931471805599453f : -INFINITY;
+      continue;
+    }
     const float inv = l_tot > 0.f ? vs / l_tot : 0.f;
     const float lse = l_tot > 0.f ? (st.m_ref + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     const size_t row = (size_t)cs.prow + (size_t)g * cs.pstride;

@@ -59,6 +59,7 @@ constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
 constexpr int kCtaMaxBatch = 1024;
 constexpr int kCtaMinTilesPerCta = 64;   // below this bound on the tiles per CTA the warp-scheduled kernel is used
 constexpr int kCtaRateMinTiles = 256;
+constexpr int kWholePairTiles = 4;       // up to this many tiles per (sequence, KV head) a pair goes to one warp whole
 inline size_t cta_rate_words(int ctas) { return 4 + 2 * (size_t)ctas; }
 
 // Launches the split-KV kernel for an FP8 (fp8 = true) or bf16 cache on `ctas` CTAs.  smem_limit[2] caches,
