@@ -193,7 +193,8 @@ PUZZLE_API puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_de
  *     free, in proportion to the speed each CTA showed in the previous large launch on this
  *     workspace; small ones (window layers, short contexts) are cut evenly over all warps, which
  *     has the shorter set-up, or not cut at all when no (sequence, KV head) can have more than
- *     four tiles (one warp then takes it whole and writes the output itself).  PUZZLE_SCHED_CTA / PUZZLE_SCHED_WARP pin one or the other
+ *     four tiles (narrow windows, very short contexts: a group of four warps, or one warp when
+ *     there are very many pairs, takes the pair whole and writes the output itself).  PUZZLE_SCHED_CTA / PUZZLE_SCHED_WARP pin one or the other
  *     (PUZZLE_SCHED_CTA needs batch <= 1024, else PUZZLE_ERR_UNSUPPORTED);
  *   workspace: device scratch of at least puzzle_decode_attn_workspace_bytes(...) bytes, 16-byte
  *     aligned, prepared once by puzzle_decode_attn_workspace_init; calls that share a workspace must

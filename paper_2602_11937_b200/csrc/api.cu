@@ -33,7 +33,7 @@ EncodeTiledFn encode_tiled() {
 struct DeviceInfo {
   int sm_count = 0;
   // per split-KV kernel (warp-scheduled FP8, bf16; tensor-memory FP8; CTA-balanced FP8, bf16); 0 = not raised yet
-  int smem_limit[6] = {0, 0, 0, 0, 0, 0};   // [5]: the multi-token kernel
+  int smem_limit[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // [5]: the multi-token kernel, [6..7]: the small-launch kernel
 };
 DeviceInfo& device_info() {
   static DeviceInfo info[64];
@@ -284,8 +284,14 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
     // Narrow windows and short contexts: with at most kWholePairTiles tiles per (sequence, KV head) a pair is not cut
     // at all.  One warp takes it whole and stores the output itself, which drops the partial, the arrival and the
     // merge (three dependent trips through L2) from a launch that is a chain of latencies anyway.
-    if (splits == 0 && tiles_per_pair_bound(desc, kv) <= kWholePairTiles) P.num_splits = 1;
-    le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
+    const bool whole_pairs = splits == 0 && tiles_per_pair_bound(desc, kv) <= kWholePairTiles;
+    if (whole_pairs && num_splits == 0 && (long long)batch * Hkv <= decode_attn_small_max_pairs(ctas)) {
+      // few pairs on top: the tiles of a pair side by side on a group of warps, combined in shared memory
+      le = launch_decode_attn_small(P, fp8, ctas, s, device_info().smem_limit + 6);
+    } else {
+      if (whole_pairs) P.num_splits = 1;
+      le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
+    }
   }
   if (le != cudaSuccess) return PUZZLE_ERR_CUDA;
   count_launch();

@@ -68,6 +68,12 @@ cudaError_t launch_decode_attn(const DecodeParams& P, bool fp8, int ctas, cudaSt
 // The CTA-balanced kernel (balanced schedule only, batch <= kCtaMaxBatch).  Its partial row blocks: one per
 // (CTA, pair) meeting, ctas + batch*Hkv at most.
 cudaError_t launch_decode_attn_cta(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit);
+// The kernel for launches in which no (sequence, KV head) has more than kWholePairTiles tiles (narrow windows, very
+// short contexts): a group of four warps per pair, one tile each, combined in shared memory; no workspace use.
+// smem_limit[2] as above.  It pays up to decode_attn_small_max_pairs(ctas) pairs; beyond, the warp-scheduled kernel
+// with one split per pair keeps its TMA rings full.
+cudaError_t launch_decode_attn_small(const DecodeParams& P, bool fp8, int ctas, cudaStream_t s, int* smem_limit);
+int decode_attn_small_max_pairs(int ctas);
 // The multi-token kernel (FP8 cache, balanced schedule): P.n_q, P.q_lens set; P.counters has one word per
 // (sequence, token pair, KV head); partial rows: decode_attn_tokens_partial_rows(...).
 cudaError_t launch_decode_attn_tokens(const DecodeParams& P, int ctas, cudaStream_t s, int* smem_limit);
