@@ -421,3 +421,33 @@ def test_stream_order_holds_next_to_kernels_of_the_caller(sched):
             assert_close(got[t], ref.reshape(got[t].shape), "step %d" % t)
     gk, gv = dev.cache_bytes()
     assert np.array_equal(gk, case["k_cache"]) and np.array_equal(gv, case["v_cache"])
+
+
+@pytest.mark.parametrize("kv_dtype", [oracle.KV_FP8_E4M3, oracle.KV_BF16], ids=["fp8", "bf16"])
+@pytest.mark.parametrize("batch,hkv", [(60, 8), (7, 1), (120, 8), (33, 4)])
+def test_launches_with_at_most_four_tiles_per_pair(batch, hkv, kv_dtype):
+    """Narrow windows and very short contexts: no (sequence, KV head) has more than four tiles, and the balanced
+    schedule does not cut pairs (a group of four warps per pair; one warp per pair when pinned to the warp-scheduled
+    kernel or when there are very many pairs: batch 120).  Lengths around every tile and block edge, empty
+    sequences, one and two rounds of pairs per group, with and without sinks, lse included."""
+    from gpu_helpers import assert_close
+    tile = 64 if kv_dtype == oracle.KV_FP8_E4M3 else 32
+    edge = [0, 1, 15, 16, 17, tile - 1, tile, tile + 1, 2 * tile - 1, 2 * tile, 2 * tile + 1, 3 * tile, 3 * tile + 5,
+            4 * tile - 1, 4 * tile, 300, 399, 400]
+    for context, windows in ((400, (3 * tile, 2 * tile, 2 * tile - 28, 1)), (4 * tile, (0, 40))):
+        lens = [min(edge[(3 * i + batch) % len(edge)], context) for i in range(batch)]
+        w = synth.Workload("narrow", 1, batch, context, [0], paged=True, hq=8 * hkv, hkv=hkv)
+        case = make_case(w, seq_lens=lens, kv_dtype=kv_dtype, poison_tail=True)
+        dev = _dev(case)
+        dev.append(); oracle_append(case)
+        for window in windows:
+            for sinks in ("case", None):
+                ref, ref_lse = oracle_attn(case, window, sinks=sinks)
+                for sched in (0, -2):                      # picked kernel, pinned warp-scheduled kernel
+                    got, lse = dev.attn(window=window, num_splits=sched, sinks=sinks)
+                    what = "context %d window %d sched %d sinks %s" % (context, window, sched, sinks)
+                    assert int(dev.status.item()) == 0, what
+                    assert_close(got, ref, what)
+                    fin = np.isfinite(ref_lse)
+                    assert np.array_equal(np.isfinite(lse), fin), what
+                    assert np.all(np.abs(lse[fin] - ref_lse[fin]) <= 2e-3), what
