@@ -492,7 +492,7 @@ NCU_CAPTURE = {
     "source": "profiles/decode_attn_cta_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "2e0db0a0b562cf407715f4b7df491eefc70ac6e936c5796374d7ca7949838c16",
+    "sha256": "c85609d7c6b631979d614468398496b96902071f881367669c93545615d0925d",
     "dram_bytes_per_launch": 1075425000 + 4126976,
 }
 
