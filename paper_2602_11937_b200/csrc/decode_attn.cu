@@ -147,10 +147,16 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_attn_kernel(const __grid_co
     cc.end = min(cc.pos + q, T);
     cc.step = 0;
   } else {
-    // consecutive units go to different SMs: a launch with fewer units than workers still uses every SM
-    cc.pos = warp * gridDim.x + blockIdx.x;
-    cc.end = P.batch * P.Hkv * P.num_splits;
-    cc.step = nW;
+    // Every worker takes one contiguous share of the units (sequence, KV head, split), shares in the order
+    // warp 0 of every CTA, warp 1 of every CTA, ...: a launch with fewer units than workers still uses every SM, and
+    // a worker meets only one or two (sequence, KV head) pairs.  (Handing units out round-robin made every worker
+    // meet many pairs; a worker that had merged one fell behind, arrived last at each of its later pairs and so
+    // had to merge those as well: with 128 splits one warp ended up with most merges of the launch.)
+    const long long units = (long long)P.batch * P.Hkv * P.num_splits;
+    const int wi = warp * gridDim.x + blockIdx.x;
+    cc.pos = (int)(wi * units / nW);
+    cc.end = (int)((wi + 1) * units / nW);
+    cc.step = 1;
   }
 
   LaneOffsets<FP8> lo;
