@@ -224,9 +224,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_attn_tc_kernel(const __gri
     cur.end = min(cur.pos + q, T);
     cur.step = 0;
   } else {
-    cur.pos = w;
-    cur.end = P.batch * Hkv * P.num_splits;
-    cur.step = nW;
+    // one contiguous share of the units per worker, shares in the order worker 0 of every CTA, worker 1 of every
+    // CTA: a worker meets one or two (sequence, KV head) pairs only (see decode_attn.cu on why not round-robin)
+    const long long units = (long long)P.batch * Hkv * P.num_splits;
+    const int wi = g * (int)gridDim.x + blockIdx.x;
+    cur.pos = (int)(wi * units / nW);
+    cur.end = (int)((wi + 1) * units / nW);
+    cur.step = 1;
   }
   Segment seg;
   auto give_up = [&]() {

@@ -82,7 +82,12 @@ __device__ __noinline__ void merge_rows(const DecodeParams& P, int b, int kvh, l
   const int total = count + count2;
   auto row_of = [&](int k) { return k < count ? base + (long long)k * kstride : base2 + (long long)(k - count) * kstride2; };
   float M = -INFINITY;
-  for (int k = c; k < total; k += 4) M = fmaxf(M, __ldcg(P.part_lse + row_of(k)));
+  for (int k = c; k < total; k += 16) {  // four loads in flight per lane: with many parts this pass is L2 round trips too
+    float l4[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) l4[j] = k + 4 * j < total ? __ldcg(P.part_lse + row_of(k + 4 * j)) : -INFINITY;
+    M = fmaxf(fmaxf(M, fmaxf(l4[0], l4[1])), fmaxf(l4[2], l4[3]));
+  }
   M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
   M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
   M = fmaxf(M, sink);
