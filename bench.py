@@ -492,8 +492,8 @@ NCU_CAPTURE = {
     "source": "profiles/decode_attn_cta_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "c85609d7c6b631979d614468398496b96902071f881367669c93545615d0925d",
-    "dram_bytes_per_launch": 1075425000 + 4126976,
+    "sha256": "de47ae32bd792bb53014a55df1d51feba755b8d872c1e7798ee22f188d763541",
+    "dram_bytes_per_launch": 1075512000 + 4117248,
 }
 
 
