@@ -257,8 +257,8 @@ def run_ours(args, plan):
         kernel_name = "decode_attn_tc_kernel (tcgen05 split-KV pass with the merge fused in)"
         dtype_name = "e4m3 tcgen05 mma on the cache codes, f32 accumulate and softmax"
     else:
-        kernel_name = ("decode_attn_cta_kernel<fp8>" if args.splits == 0 else "decode_attn_kernel<fp8>") + \
-            " (split-KV pass with the merge fused in)"
+        kernel_name = "%s<%s> (split-KV pass with the merge fused in)" % (
+            P.puzzle_decode_attn_kernel_name(desc, views[0], w.batch, args.splits), "fp8")
         dtype_name = "f16 mma on e4m3 codes, f32 accumulate and softmax"
     ws = torch.empty(P.puzzle_decode_attn_workspace_bytes(desc, w.batch, args.splits), dtype=torch.uint8, device=dev)
     P.puzzle_decode_attn_workspace_init(desc, w.batch, ws)
@@ -492,7 +492,7 @@ NCU_CAPTURE = {
     "source": "profiles/decode_attn_cta_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "de47ae32bd792bb53014a55df1d51feba755b8d872c1e7798ee22f188d763541",
+    "sha256": "b772f07d3cf28e7bd44b13ed00b7b168dffcc45f541718d53af270f88eeede44",
     "dram_bytes_per_launch": 1075512000 + 4117248,
 }
 

@@ -366,6 +366,16 @@ PUZZLE_API puzzle_status puzzle_hbm_read_probe(const void* buf, size_t bytes, ui
 /* Static description of a status code (host string, never NULL). */
 PUZZLE_API const char* puzzle_status_string(puzzle_status s);
 
+/* Which of the library's kernels puzzle_decode_attn would launch for these
+ * arguments ("decode_attn_cta_kernel", "decode_attn_kernel",
+ * "decode_attn_small_kernel"; host string, never NULL; "invalid arguments" when
+ * the call would be refused).  The choice follows from desc, the batch, the
+ * width of a block-table row and num_splits alone, so nothing is launched or
+ * read on the device.  For logs and benchmarks that name what they time; the
+ * paper has no counterpart (it does not describe kernels). */
+PUZZLE_API const char* puzzle_decode_attn_kernel_name(const puzzle_layer_desc* desc, const puzzle_kv_view* kv,
+                                                      int32_t batch, int32_t num_splits);
+
 /* Number of kernels this library has launched from this process so far. */
 PUZZLE_API int64_t puzzle_launch_count(void);
 

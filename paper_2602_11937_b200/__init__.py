@@ -40,6 +40,7 @@ from .binding import (  # noqa: F401
     puzzle_kv_append_tokens,
     puzzle_kv_scales_from_amax,
     puzzle_launch_count,
+    puzzle_decode_attn_kernel_name,
     puzzle_status_string,
 )
 from .stack import DecodeStack  # noqa: F401,E402

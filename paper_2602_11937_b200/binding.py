@@ -40,6 +40,7 @@ EXPORTS = (
     "puzzle_hbm_read_probe",
     "puzzle_status_string",
     "puzzle_launch_count",
+    "puzzle_decode_attn_kernel_name",
 )
 
 
@@ -121,6 +122,8 @@ def _load():
         lib.puzzle_status_string.argtypes = [ctypes.c_int]
         lib.puzzle_launch_count.restype = ctypes.c_int64
         lib.puzzle_launch_count.argtypes = []
+        lib.puzzle_decode_attn_kernel_name.restype = ctypes.c_char_p
+        lib.puzzle_decode_attn_kernel_name.argtypes = [vp, vp, i32, i32]
         _lib = lib
     return _lib
 
@@ -178,6 +181,11 @@ def puzzle_status_string(code: int) -> str:
 
 def puzzle_launch_count() -> int:
     return int(_load().puzzle_launch_count())
+
+
+def puzzle_decode_attn_kernel_name(desc: "LayerDesc", kv: "KVView", batch: int, num_splits: int = 0) -> str:
+    return _load().puzzle_decode_attn_kernel_name(ctypes.byref(desc), ctypes.byref(kv), int(batch),
+                                                  int(num_splits)).decode()
 
 
 def _check(code: int, where: str):

@@ -124,7 +124,28 @@ long long tiles_per_pair_bound(const puzzle_layer_desc* d, const puzzle_kv_view*
 bool use_cta_kernel(const puzzle_layer_desc* d, const puzzle_kv_view* kv, int batch, int num_splits) {
   if (num_splits == PUZZLE_SCHED_CTA) return true;
   if (num_splits != 0 || batch > kCtaMaxBatch) return false;
-  return tiles_per_pair_bound(d, kv) * batch * d->num_kv_heads >= (long long)kCtaMinTilesPerCta * grid_ctas();
+  // What the CTA-balanced kernel wins (no tail, CTAs cut by speed) grows with the length of the launch and of the
+  // pairs; what it costs (a longer set-up, a claim and a hand-over per piece) weighs most on many short pairs.
+  // Measured crossovers, in tiles per CTA: 64 with pairs of 256 tiles or more, about 200 at 128 tiles per pair,
+  // about 600 below.
+  const long long per_pair = tiles_per_pair_bound(d, kv);
+  const long long min_per_cta = per_pair >= 256 ? kCtaMinTilesPerCta : (per_pair >= 128 ? 200 : 600);
+  return per_pair * batch * d->num_kv_heads >= min_per_cta * grid_ctas();
+}
+
+// The kernel a call of puzzle_decode_attn runs on.
+enum class Kernel { kCta, kWarp, kWarpWholePairs, kSmall };
+Kernel pick_kernel(const puzzle_layer_desc* d, const puzzle_kv_view* kv, int batch, int num_splits) {
+  if (use_cta_kernel(d, kv, batch, num_splits)) return Kernel::kCta;
+  // Narrow windows and short contexts: with at most kWholePairTiles tiles per (sequence, KV head) a pair is not cut
+  // at all.  A group of four warps (few pairs) or one warp (many pairs, or the warp-scheduled kernel pinned) takes
+  // it whole and stores the output itself, which drops the partial, the arrival and the merge (three dependent
+  // trips through L2) from a launch that is a chain of latencies anyway.
+  const bool whole_pairs = num_splits <= 0 && tiles_per_pair_bound(d, kv) <= kWholePairTiles;
+  if (!whole_pairs) return Kernel::kWarp;
+  if (num_splits == 0 && (long long)batch * d->num_kv_heads <= decode_attn_small_max_pairs(grid_ctas()))
+    return Kernel::kSmall;
+  return Kernel::kWarpWholePairs;
 }
 
 size_t workspace_floats(int batch, int Hkv, int num_splits, int kv_dtype) {
@@ -175,6 +196,17 @@ const char* puzzle_status_string(puzzle_status s) {
 }
 
 int64_t puzzle_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* puzzle_decode_attn_kernel_name(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, int32_t batch,
+                                           int32_t num_splits) {
+  if (check_desc(desc) != PUZZLE_OK || !kv || batch <= 0 || batch > kMaxBatch || num_splits < PUZZLE_SCHED_WARP)
+    return "invalid arguments";
+  switch (pick_kernel(desc, kv, batch, num_splits)) {
+    case Kernel::kCta: return "decode_attn_cta_kernel";
+    case Kernel::kSmall: return "decode_attn_small_kernel";
+    default: return "decode_attn_kernel";
+  }
+}
 
 puzzle_status puzzle_kv_append(const puzzle_layer_desc* desc, const puzzle_kv_view* kv, const void* k_new,
                                const void* v_new, int32_t batch, int32_t* dev_status, void* stream) {
@@ -278,19 +310,20 @@ static puzzle_status decode_attn_impl(const puzzle_layer_desc* desc, const puzzl
   cudaError_t le;
   if (tc) {
     le = launch_decode_attn_tc(P, ctas, s, device_info().smem_limit + 2);
-  } else if (use_cta_kernel(desc, kv, batch, num_splits)) {
-    le = launch_decode_attn_cta(P, fp8, ctas, s, device_info().smem_limit + 3);
   } else {
-    // Narrow windows and short contexts: with at most kWholePairTiles tiles per (sequence, KV head) a pair is not cut
-    // at all.  One warp takes it whole and stores the output itself, which drops the partial, the arrival and the
-    // merge (three dependent trips through L2) from a launch that is a chain of latencies anyway.
-    const bool whole_pairs = splits == 0 && tiles_per_pair_bound(desc, kv) <= kWholePairTiles;
-    if (whole_pairs && num_splits == 0 && (long long)batch * Hkv <= decode_attn_small_max_pairs(ctas)) {
-      // few pairs on top: the tiles of a pair side by side on a group of warps, combined in shared memory
-      le = launch_decode_attn_small(P, fp8, ctas, s, device_info().smem_limit + 6);
-    } else {
-      if (whole_pairs) P.num_splits = 1;
-      le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
+    switch (pick_kernel(desc, kv, batch, num_splits)) {
+      case Kernel::kCta:
+        le = launch_decode_attn_cta(P, fp8, ctas, s, device_info().smem_limit + 3);
+        break;
+      case Kernel::kSmall:
+        le = launch_decode_attn_small(P, fp8, ctas, s, device_info().smem_limit + 6);
+        break;
+      case Kernel::kWarpWholePairs:
+        P.num_splits = 1;
+        le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
+        break;
+      default:
+        le = launch_decode_attn(P, fp8, ctas, s, device_info().smem_limit);
     }
   }
   if (le != cudaSuccess) return PUZZLE_ERR_CUDA;

@@ -57,7 +57,7 @@ constexpr int kDecodeWarpsBf16 = 12, kDecodeStagesBf16 = 2, kTileBf16 = 32;
 // CTA slot at the start of the workspace (before the arrival counters: a CTA counter, the buffer switch, two pad words, then two
 // float buffers of one speed per CTA) and are cut by the speeds the launch before them noted.
 constexpr int kCtaMaxBatch = 1024;
-constexpr int kCtaMinTilesPerCta = 64;   // below this bound on the tiles per CTA the warp-scheduled kernel is used
+constexpr int kCtaMinTilesPerCta = 64;   // below this bound on the tiles per CTA the warp-scheduled kernel is used (more with short pairs)
 constexpr int kCtaRateMinTiles = 256;
 constexpr int kWholePairTiles = 4;       // up to this many tiles per (sequence, KV head) a pair goes to one warp whole
 inline size_t cta_rate_words(int ctas) { return 4 + 2 * (size_t)ctas; }

@@ -451,3 +451,31 @@ def test_launches_with_at_most_four_tiles_per_pair(batch, hkv, kv_dtype):
                     fin = np.isfinite(ref_lse)
                     assert np.array_equal(np.isfinite(lse), fin), what
                     assert np.all(np.abs(lse[fin] - ref_lse[fin]) <= 2e-3), what
+
+
+def test_kernel_choice_follows_the_shape_of_the_launch():
+    """puzzle_decode_attn_kernel_name says what puzzle_decode_attn would launch; the choice uses the host's bounds
+    only (batch, width of a block-table row, window).  148 SMs assumed for the sizes in the middle."""
+    import paper_2602_11937_b200 as P
+    if torch.cuda.get_device_properties(0).multi_processor_count != 148:
+        pytest.skip("thresholds are in tiles per SM; the cases below are sized for 148 SMs")
+    dummy = torch.zeros(1, 8, 16, 64, dtype=torch.uint8, device="cuda")
+    lens = torch.zeros(4096, dtype=torch.int32, device="cuda")
+
+    def name(batch, context, window=0, splits=0):
+        v = P.kv_view(dummy, dummy, lens, max_blocks_per_seq=(context + 15) // 16)
+        return P.puzzle_decode_attn_kernel_name(P.layer_desc(window=window), v, batch, splits)
+
+    assert name(16, 65536) == "decode_attn_cta_kernel"              # the 64K workload
+    assert name(8, 16384) == "decode_attn_cta_kernel"               # mid-size launch, long pairs
+    assert name(128, 1024) == "decode_attn_kernel"                  # the same bytes in many short pairs
+    assert name(1024, 1024) == "decode_attn_cta_kernel"             # ... unless the launch is large
+    assert name(4, 1024) == "decode_attn_kernel"                    # a small launch
+    assert name(64, 40000, window=128) == "decode_attn_small_kernel"   # narrow window, few pairs
+    assert name(200, 40000, window=128) == "decode_attn_kernel"     # narrow window, many pairs: one warp per pair
+    assert name(64, 40000, window=8192) == "decode_attn_cta_kernel"
+    assert name(2, 200) == "decode_attn_small_kernel"               # very short contexts
+    assert name(16, 65536, splits=8) == "decode_attn_kernel"        # explicit splits
+    assert name(4, 1024, splits=P.SCHED_CTA) == "decode_attn_cta_kernel"
+    assert name(2, 200, splits=P.SCHED_WARP) == "decode_attn_kernel"
+    assert name(0, 1024) == "invalid arguments" and name(4, 1024, splits=-3) == "invalid arguments"
