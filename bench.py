@@ -492,8 +492,8 @@ NCU_CAPTURE = {
     "source": "profiles/decode_attn_cta_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "b772f07d3cf28e7bd44b13ed00b7b168dffcc45f541718d53af270f88eeede44",
-    "dram_bytes_per_launch": 1075512000 + 4117248,
+    "sha256": "9df0d4b71b68352bab7afa5aa76b409bc5cc8ccf1f75ababcec441fc07f84d6f",
+    "dram_bytes_per_launch": 1075519000 + 4436736,
 }
 
 

@@ -136,8 +136,16 @@ __device__ __noinline__ void claim_tiles(uint32_t ctl_a, const DecodeParams& P, 
       return;
     }
     if (pos < c0.x || pos >= c0.y) {  // another pair than last time
-      const int b = seq_of(cum, P.batch, pos);
-      const SeqTiles q = seq_tiles<TT>(P, b);
+      int b = c0.z;
+      SeqTiles q;
+      if (c0.y > c0.x && pos >= cum[b] && pos < cum[b + 1]) {
+        // another KV head of the same sequence (seven pair changes in eight): its lengths are known, and neither
+        // the search nor the trip to global memory for the length stands between this warp and its next copies
+        q.nt = c0.y - c0.x; q.tlo = c1.x; q.L = c1.y; q.lo = c1.z;
+      } else {
+        b = seq_of(cum, P.batch, pos);
+        q = seq_tiles<TT>(P, b);
+      }
       const int kvh = (pos - cum[b]) / q.nt;
       c0 = make_int4(cum[b] + kvh * q.nt, cum[b] + (kvh + 1) * q.nt, b, kvh);
       c1 = make_int4(q.tlo, q.L, q.lo, 0);
