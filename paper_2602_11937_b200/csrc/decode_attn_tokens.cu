@@ -5,8 +5,8 @@
 // The bytes of a step do not grow with the number of query tokens, only the arithmetic does, so query tokens are
 // processed in pairs that share one pass over the K/V tiles: in the single-token kernels rows 8-15 of the
 // S^T = Q.K^T MMA are empty; here they carry the eight heads of a second query token, so the tile's E4M3 -> f16
-// converts and its S MMAs serve both tokens, and only the softmax and the P.V MMAs are paid per token (P.V with
-// the same converted V fragments).  A pair of tokens (2j, 2j+1) of sequence b is one row of the schedule; a
+// converts and its S MMAs serve both tokens, and only the softmax and half of the P.V MMAs are paid per token
+// (P.V with the same converted V fragments).  A pair of tokens (2j, 2j+1) of sequence b is one row of the schedule; a
 // causal mask gives the earlier token one key fewer (and a window that starts one key earlier).  An odd last
 // token is paired with itself.  Sequences with more than two new tokens take several rows, whose repeated reads
 // of the same blocks are neighbours in the schedule and are served by L2.
@@ -14,7 +14,9 @@
 // Everything else is the warp-scheduled kernel's design (decode_attn.cu): every warp an independent worker with
 // a private ring of TMA stages, the tile space of all rows cut evenly over the workers, one float32 partial
 // (o, lse) per (worker, row, KV head) and query head, merged by the worker whose arrival completes the (row, KV
-// head).  Eight warps of 255 registers instead of twelve of 168: two tokens' accumulators need the room.
+// head).  Twelve warps of two stages, as there: the two tokens share one accumulator (see TileState2), which
+// brings the kernel to 168 registers with a few spilled words outside the MMA stream; eight warps of three stages
+// (190 registers, no spill) measured 5 % slower on two tokens and 10 % slower on four.
 #include <cuda.h>
 
 #include <climits>
@@ -26,7 +28,7 @@
 namespace puzzle {
 namespace {
 
-constexpr int kTokWarps = 8, kTokStages = 3, kTokTile = 64;
+constexpr int kTokWarps = 12, kTokStages = 2, kTokTile = 64;
 constexpr int kPairRows = 2 * kGroup;  // partial rows per (worker, row, KV head): 8 heads of each of the two tokens
 
 // One row of the schedule: query tokens t0 and t1 (= t0 + 1, or t0 again for an odd last token) of sequence b.
@@ -90,21 +92,23 @@ __device__ __forceinline__ bool next_tok_segment(int& pos, int end, TokSegment& 
 }
 
 // Running state of a warp over the tiles of one (row, KV head): as TileState in decode_tile.cuh, for two query
-// tokens.  Token A (t0) sits on MMA rows 0-7, token B (t1) on rows 8-15 of S; each has its own logit scale,
-// reference maximum, row sum and accumulator.
+// tokens.  Token A (t0) sits on MMA rows 0-7, token B (t1) on rows 8-15 of S and of O; each has its own logit
+// scale, reference maximum and row sum.  P.V runs twice per V fragment, with A = [P_A ; P_B] of the high terms and
+// of the low terms of the exact two-term f16 split of P, both into the same accumulator (the single-token kernels
+// put the low terms on rows 8-15 instead and add the two halves at the end).
 struct TileState2 {
   uint32_t qa[4][4];
   float alpha[2], m_ref[2], l_run[2];
-  float O[2][8][4];
+  float O[8][4];   // O[dim n-tile][token A: cols 2c, 2c+1 | token B: cols 2c, 2c+1] (rows g and g + 8 of the MMA)
 
   __device__ __forceinline__ void reset() {
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
       m_ref[t] = -INFINITY;
       l_run[t] = 0.f;
-#pragma unroll
-      for (int nd = 0; nd < 8; ++nd) O[t][nd][0] = O[t][nd][1] = O[t][nd][2] = O[t][nd][3] = 0.f;
     }
+#pragma unroll
+    for (int nd = 0; nd < 8; ++nd) O[nd][0] = O[nd][1] = O[nd][2] = O[nd][3] = 0.f;
   }
 
   // Query row of token `tok` (head g of the group, 64 bf16), scaled by a power of two into f16 exactly; see
@@ -173,8 +177,10 @@ struct TileState2 {
         }
       }
     }
-    // ---- online softmax per token, then that token's P.V
-    uint32_t pa[2][NB][4];
+    // ---- online softmax per token.  P is split exactly into a high and a low f16 term; both terms of both tokens
+    // go through the same accumulator rows: A = [P_A ; P_B] (rows 0-7 | 8-15), once with the high and once with
+    // the low terms, so O needs the registers of one token's two-term accumulator
+    uint32_t pa_hi[NB][4], pa_lo[NB][4];
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
       float mx = -INFINITY;
@@ -188,9 +194,7 @@ struct TileState2 {
           const float corr = ex2(m_ref[t] - mx);
           l_run[t] *= corr;
 #pragma unroll
-          for (int nd = 0; nd < 8; ++nd) {
-            O[t][nd][0] *= corr; O[t][nd][1] *= corr; O[t][nd][2] *= corr; O[t][nd][3] *= corr;
-          }
+          for (int nd = 0; nd < 8; ++nd) { O[nd][2 * t] *= corr; O[nd][2 * t + 1] *= corr; }
           m_ref[t] = mx;
         }
       }
@@ -204,8 +208,8 @@ struct TileState2 {
           l_run[t] += p0 + p1;
           const float h0 = __uint_as_float(__float_as_uint(p0) & 0xffffe000u);
           const float h1 = __uint_as_float(__float_as_uint(p1) & 0xffffe000u);
-          pa[t][blk][2 * u + 0] = f32x2_to_f16x2(h0, h1);
-          pa[t][blk][2 * u + 1] = f32x2_to_f16x2(p0 - h0, p1 - h1);
+          pa_hi[blk][2 * u + t] = f32x2_to_f16x2(h0, h1);
+          pa_lo[blk][2 * u + t] = f32x2_to_f16x2(p0 - h0, p1 - h1);
         }
       }
     }
@@ -228,26 +232,24 @@ struct TileState2 {
         uint32_t r0, r1, r2, r3;
         ldsm_x2_trans_b8(vb[ch] + blk2 * 2 * BLOCK_BYTES, r0, r1, r2, r3);
         if constexpr (EDGE) { r0 &= mlo; r1 &= mlo; r2 &= mhi; r3 &= mhi; }
-        uint32_t b0, b1;
+        // two independent accumulators alternate, so that an MMA never waits for the one issued just before it
+        uint32_t b0, b1, d0, d1;
         e4m3x4_to_f16x2x2(r0, b0, b1);
-#pragma unroll
-        for (int t = 0; t < 2; ++t)
-          mma_f16(O[t][2 * ch], pa[t][2 * blk2][0], pa[t][2 * blk2][1], pa[t][2 * blk2][2], pa[t][2 * blk2][3], b0, b1);
-        e4m3x4_to_f16x2x2(r1, b0, b1);
-#pragma unroll
-        for (int t = 0; t < 2; ++t)
-          mma_f16(O[t][2 * ch + 1], pa[t][2 * blk2][0], pa[t][2 * blk2][1], pa[t][2 * blk2][2], pa[t][2 * blk2][3], b0,
-                  b1);
+        e4m3x4_to_f16x2x2(r1, d0, d1);
+        mma_f16(O[2 * ch], pa_hi[2 * blk2][0], pa_hi[2 * blk2][1], pa_hi[2 * blk2][2], pa_hi[2 * blk2][3], b0, b1);
+        mma_f16(O[2 * ch + 1], pa_hi[2 * blk2][0], pa_hi[2 * blk2][1], pa_hi[2 * blk2][2], pa_hi[2 * blk2][3], d0, d1);
+        mma_f16(O[2 * ch], pa_lo[2 * blk2][0], pa_lo[2 * blk2][1], pa_lo[2 * blk2][2], pa_lo[2 * blk2][3], b0, b1);
+        mma_f16(O[2 * ch + 1], pa_lo[2 * blk2][0], pa_lo[2 * blk2][1], pa_lo[2 * blk2][2], pa_lo[2 * blk2][3], d0, d1);
         e4m3x4_to_f16x2x2(r2, b0, b1);
-#pragma unroll
-        for (int t = 0; t < 2; ++t)
-          mma_f16(O[t][2 * ch], pa[t][2 * blk2 + 1][0], pa[t][2 * blk2 + 1][1], pa[t][2 * blk2 + 1][2],
-                  pa[t][2 * blk2 + 1][3], b0, b1);
-        e4m3x4_to_f16x2x2(r3, b0, b1);
-#pragma unroll
-        for (int t = 0; t < 2; ++t)
-          mma_f16(O[t][2 * ch + 1], pa[t][2 * blk2 + 1][0], pa[t][2 * blk2 + 1][1], pa[t][2 * blk2 + 1][2],
-                  pa[t][2 * blk2 + 1][3], b0, b1);
+        e4m3x4_to_f16x2x2(r3, d0, d1);
+        mma_f16(O[2 * ch], pa_hi[2 * blk2 + 1][0], pa_hi[2 * blk2 + 1][1], pa_hi[2 * blk2 + 1][2],
+                pa_hi[2 * blk2 + 1][3], b0, b1);
+        mma_f16(O[2 * ch + 1], pa_hi[2 * blk2 + 1][0], pa_hi[2 * blk2 + 1][1], pa_hi[2 * blk2 + 1][2],
+                pa_hi[2 * blk2 + 1][3], d0, d1);
+        mma_f16(O[2 * ch], pa_lo[2 * blk2 + 1][0], pa_lo[2 * blk2 + 1][1], pa_lo[2 * blk2 + 1][2],
+                pa_lo[2 * blk2 + 1][3], b0, b1);
+        mma_f16(O[2 * ch + 1], pa_lo[2 * blk2 + 1][0], pa_lo[2 * blk2 + 1][1], pa_lo[2 * blk2 + 1][2],
+                pa_lo[2 * blk2 + 1][3], d0, d1);
       }
     }
   }
@@ -458,7 +460,7 @@ __global__ void __launch_bounds__(kTokWarps * 32, 1) decode_attn_tokens_kernel(c
 #pragma unroll
       for (int nd = 0; nd < 8; ++nd)
         *reinterpret_cast<float2*>(po + 8 * nd) =
-            make_float2((st.O[t][nd][0] + st.O[t][nd][2]) * inv, (st.O[t][nd][1] + st.O[t][nd][3]) * inv);
+            make_float2(st.O[nd][2 * t] * inv, st.O[nd][2 * t + 1] * inv);
       if (c == 0) P.part_lse[row] = l_tot > 0.f ? (st.m_ref[t] + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     }
     // ---- arrival; the warp that completes the (row, KV head) merges it and leaves the counter at zero
