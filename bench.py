@@ -702,6 +702,73 @@ def run_reference(args):
     }))
 
 
+def run_tokens(args):
+    """A decode step with --tokens N new tokens per sequence on workload 3 (a multi-token step, or a chunk of a
+    prompt): bulk append of the N tokens + causal attention of the N query tokens by puzzle_decode_attn_tokens,
+    timed with CUDA events over regions of --steps steps, beside the one-token step on the same caches.  Prints its
+    own JSON line (not the headline metric)."""
+    import paper_2602_11937_b200 as P
+    import statistics
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = synth.workload(args.config)
+    n_q = args.tokens
+    layers = [build_layer(w, l, dev) for l in range(args.layers)]
+    seq_lens = synth.draw_seq_lens(w).to(dev)
+    desc = P.layer_desc(num_q_heads=w.hq, num_kv_heads=w.hkv, head_dim=w.head_dim, block_size=w.block)
+    views = [P.kv_view(L["k_cache"], L["v_cache"], seq_lens, block_table=L["table"],
+                       max_blocks_per_seq=w.blocks_per_seq, k_scale=L["k_scale"], v_scale=L["v_scale"]) for L in layers]
+    g = torch.Generator(device=dev).manual_seed(0x5EED0000 + 77)
+    q = torch.randn(w.batch, n_q, w.hq, w.head_dim, generator=g, device=dev).to(torch.bfloat16)
+    k_new = torch.randn(w.batch, n_q, w.hkv, w.head_dim, generator=g, device=dev).to(torch.bfloat16)
+    v_new = torch.randn(w.batch, n_q, w.hkv, w.head_dim, generator=g, device=dev).to(torch.bfloat16)
+    sinks = synth.draw_sinks(w, 0, dev)
+    out = torch.empty_like(q)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.zeros(P.puzzle_decode_attn_tokens_workspace_bytes(desc, w.batch, n_q), dtype=torch.uint8, device=dev)
+    P.puzzle_decode_attn_tokens_workspace_init(desc, w.batch, n_q, ws)
+    ws1 = torch.zeros(P.puzzle_decode_attn_workspace_bytes(desc, w.batch, 0), dtype=torch.uint8, device=dev)
+    P.puzzle_decode_attn_workspace_init(desc, w.batch, ws1)
+    q1, k1, v1, out1 = q[:, 0].contiguous(), k_new[:, 0].contiguous(), v_new[:, 0].contiguous(), out[:, 0].contiguous()
+
+    def step_tokens(i):
+        P.puzzle_kv_append_tokens(desc, views[i % len(views)], k_new, v_new, None, dev_status=status)
+        P.puzzle_decode_attn_tokens(desc, views[i % len(views)], q, sinks, out, workspace=ws, dev_status=status)
+
+    def step_one(i):
+        P.puzzle_kv_append(desc, views[i % len(views)], k1, v1, dev_status=status)
+        P.puzzle_decode_attn(desc, views[i % len(views)], q1, sinks, out1, None, workspace=ws1, dev_status=status)
+
+    def timed(step):
+        for i in range(max(3, args.warmup)):
+            step(i)
+        torch.cuda.synchronize()
+        regions = []
+        while len(regions) < 3 or (sum(regions) < args.min_seconds * 1e3 and len(regions) < args.max_regions):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(args.steps):
+                step(i)
+            b.record()
+            torch.cuda.synchronize()
+            regions.append(a.elapsed_time(b))
+        return statistics.median(regions) / args.steps * 1e3
+
+    us_one = timed(step_one)
+    us_tok = timed(step_tokens)
+    lens = seq_lens.tolist()
+    nbytes = algorithmic_bytes(w, lens, 0)
+    print(json.dumps({
+        "metric": "multi_token_decode_step", "workload": w.name, "query_tokens_per_sequence": n_q,
+        "us_per_step": round(us_tok, 2), "us_per_one_token_step": round(us_one, 2),
+        "ratio_to_one_token_step": round(us_tok / us_one, 3), "steps": args.steps,
+        "kv_gbs": round(nbytes / (us_tok * 1e-6) / 1e9, 1),
+        "l2": "%d layer caches of %.0f MiB rotated (larger than L2)" % (len(layers), nbytes / 2 ** 20),
+        "kernel": "decode_attn_tokens_kernel (pairs of query tokens share one pass over the K/V tiles)",
+        "dev_status": int(status.item())}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -723,6 +790,8 @@ def main():
                     help="instead of the headline run: one step of the 36-layer stack of workload 4 or 5")
     ap.add_argument("--study", default=None, choices=["scales"],
                     help="instead of the headline run: FP8 KV with, with power-of-two and without scales on synthetic streams")
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="instead of the headline run: a step with this many new tokens per sequence (multi-token kernel)")
     ap.add_argument("--pattern", default="parent", choices=["parent", "every4th", "selective"])
     ap.add_argument("--kv", default="fp8", choices=["fp8", "bf16"])
     ap.add_argument("--kernel", default="mma", choices=["mma", "tcgen05"],
@@ -740,6 +809,8 @@ def main():
         sys.exit(spawn_ranks(args.gpus))
     if args.study:
         run_study(args)
+    elif args.tokens:
+        run_tokens(args)
     elif args.stack:
         run_stack(args)
     elif args.impl == "reference":
