@@ -187,15 +187,17 @@ PUZZLE_API puzzle_status puzzle_decode_attn_workspace_init(const puzzle_layer_de
  *   q: bf16 [batch][num_q_heads][head_dim], 8-byte aligned;  sinks: float32 [num_q_heads] or NULL (no sink);
  *   out: bf16 [batch][num_q_heads][head_dim], 16-byte aligned;  lse_out: float32 [batch][num_q_heads] or NULL;
  *   num_splits: 0 = balanced schedule (recommended); S >= 1 = every (sequence, KV head) context is
- *     cut into S equal runs of 64-token tiles.  The balanced schedule has two kernels and picks by
- *     what the host knows about the size of the launch (batch, window, block-table row length):
- *     large launches are cut into one range of tiles per CTA, handed out to its warps as they become
- *     free, in proportion to the speed each CTA showed in the previous large launch on this
- *     workspace; small ones (window layers, short contexts) are cut evenly over all warps, which
- *     has the shorter set-up, or not cut at all when no (sequence, KV head) can have more than
- *     four tiles (narrow windows, very short contexts: a group of four warps, or one warp when
- *     there are very many pairs, takes the pair whole and writes the output itself).  PUZZLE_SCHED_CTA / PUZZLE_SCHED_WARP pin one or the other
- *     (PUZZLE_SCHED_CTA needs batch <= 1024, else PUZZLE_ERR_UNSUPPORTED);
+ *     cut into S equal runs of 64-token tiles.  The balanced schedule has three kernels and picks by
+ *     what the host knows about the size of the launch (batch, window, block-table row length;
+ *     puzzle_decode_attn_kernel_name tells which): large launches are cut into one range of tiles
+ *     per CTA, handed out to its warps as they become free, in proportion to the speed each CTA
+ *     showed in the previous large launch on this workspace; smaller ones, and mid-size ones made
+ *     of many short contexts, are cut evenly over all warps, which has the shorter set-up; and
+ *     when no (sequence, KV head) can have more than four tiles (narrow windows, very short
+ *     contexts) nothing is cut: a group of four warps, or one warp when there are very many
+ *     pairs, takes the pair whole and writes the output itself.  PUZZLE_SCHED_CTA and
+ *     PUZZLE_SCHED_WARP pin the first or the second kernel (PUZZLE_SCHED_CTA needs batch <= 1024,
+ *     else PUZZLE_ERR_UNSUPPORTED);
  *   workspace: device scratch of at least puzzle_decode_attn_workspace_bytes(...) bytes, 16-byte
  *     aligned, prepared once by puzzle_decode_attn_workspace_init; calls that share a workspace must
  *     not overlap on the GPU.  Besides partials and counters it keeps the CTA speeds between calls:
