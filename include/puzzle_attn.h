@@ -27,7 +27,11 @@
  *     kernel of the library reads or writes global memory only after all
  *     earlier work on its stream has completed (some are launched so that
  *     their thread blocks are placed, and set up shared memory, while the
- *     kernel before them drains; nothing else runs early).
+ *     kernel before them drains; nothing else runs early).  The decode kernels
+ *     in turn let a following kernel be placed early IF that kernel was
+ *     launched with programmatic stream serialization; such a kernel must, as
+ *     that attribute always requires, wait for its grid dependency before it
+ *     reads what the library wrote.  Ordinary launches are unaffected.
  *   - The balanced schedule hands tiles of the cache to warps as they become
  *     free, so the order of the float32 sums can differ between two calls on the
  *     same inputs: outputs agree to rounding (the last bit of a bf16 value may
