@@ -492,7 +492,7 @@ NCU_CAPTURE = {
     "source": "profiles/decode_attn_cta_fp8_c3_64k_ncu_full.md (one launch, ncu --set full --clock-control none)",
     "workload": 3, "kernel": "mma", "splits": 0,
     "sources": ("decode_attn_cta.cu", "decode_tile.cuh", "decode_sched.cuh", "common.cuh", "decode_attn.cuh"),
-    "sha256": "9df0d4b71b68352bab7afa5aa76b409bc5cc8ccf1f75ababcec441fc07f84d6f",
+    "sha256": "1cf92a3f269d5ab74de65037e8c0d3bfb2b26a0a6e2d4063e2953d2c8809e362",
     "dram_bytes_per_launch": 1075519000 + 4436736,
 }
 

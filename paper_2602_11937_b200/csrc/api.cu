@@ -239,12 +239,13 @@ puzzle_status puzzle_kv_append_tokens(const puzzle_layer_desc* desc, const puzzl
   const long long per_seq = (long long)n_new * desc->num_kv_heads * (kHeadDim / 8);
   if (per_seq > 0x7fffffffll || batch > 65535) return PUZZLE_ERR_SHAPE;
   const dim3 grid((unsigned)((per_seq + 255) / 256), (unsigned)batch, 2);
-  kv_append_tokens_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      kv->k_cache, kv->v_cache, static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), new_lens,
-      kv->block_table, kv->seq_lens, kv->k_scale, kv->v_scale, kv->num_blocks, batch, n_new, desc->num_kv_heads,
-      kv->max_blocks_per_seq, desc->kv_dtype, dev_status);
+  const cudaError_t e = launch_dependent(
+      kv_append_tokens_kernel, grid, dim3(256), 0, static_cast<cudaStream_t>(stream), kv->k_cache, kv->v_cache,
+      static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), new_lens, kv->block_table, kv->seq_lens,
+      kv->k_scale, kv->v_scale, kv->num_blocks, batch, n_new, desc->num_kv_heads, kv->max_blocks_per_seq,
+      desc->kv_dtype, dev_status);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
+  return e == cudaSuccess ? PUZZLE_OK : PUZZLE_ERR_CUDA;
 }
 
 size_t puzzle_decode_attn_workspace_bytes(const puzzle_layer_desc* desc, int32_t batch, int32_t num_splits) {

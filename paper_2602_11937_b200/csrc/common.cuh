@@ -20,7 +20,7 @@ constexpr int kMaxBatch = 4096;
 void count_launch();
 
 // --------------------------------------------- programmatic dependent launch --
-// The append and the two balanced decode kernels are launched so that their CTAs may be placed on an SM as soon as
+// The append kernels and the mma.sync decode kernels are launched so that their CTAs may be placed on an SM as soon as
 // the kernel before them on the stream lets go of it, instead of after that whole grid has drained and a launch
 // latency on top.  A kernel launched this way calls grid_dependency_wait() before its first access to global memory:
 // it returns once every earlier kernel on the stream has completed and its writes are visible, so nothing the caller

@@ -334,6 +334,8 @@ __global__ void __launch_bounds__(kTokWarps * 32, 1) decode_attn_tokens_kernel(c
     tma_prefetch_desc(&P.tmK);
     tma_prefetch_desc(&P.tmV);
   }
+  release_dependents();
+  grid_dependency_wait();   // nothing above reads or writes global memory
   // ---- schedule: tiles of every row, prefix sums
   for (int r = threadIdx.x; r < rows; r += blockDim.x) {
     const RowInfo i = row_info(P, r);
@@ -521,8 +523,7 @@ cudaError_t launch_decode_attn_tokens(const DecodeParams& P, int ctas, cudaStrea
   const size_t need = 1024 + (size_t)kTokWarps * kTokStages * 2 * (kTokTile / kBlock) * kBlock * kHeadDim +
                       kTokWarps * kTokStages * 8 + (size_t)(rows + 1) * sizeof(int);
   if (need > (size_t)*smem_limit) return cudaErrorInvalidValue;  // too many rows for the schedule array
-  decode_attn_tokens_kernel<<<ctas, kTokWarps * 32, need, s>>>(P);
-  return cudaGetLastError();
+  return launch_dependent(decode_attn_tokens_kernel, dim3(ctas), dim3(kTokWarps * 32), need, s, P);
 }
 
 }  // namespace puzzle

@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(256) kv_append_tokens_kernel(void* k_cache, vo
                                                                long long num_blocks, int batch, int n_new, int Hkv,
                                                                int max_blocks_per_seq, int kv_dtype,
                                                                int32_t* dev_status) {
+  grid_dependency_wait();              // no early release, for the reason given in kv_append_kernel
   constexpr int kOct = kHeadDim / 8;   // 16-byte pieces per (token, head) row
   // grid: x over the (token, head, piece) of one sequence, y = sequence, z = K or V
   const int per_seq = n_new * Hkv * kOct;
